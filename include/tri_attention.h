@@ -1,0 +1,175 @@
+/*
+ * tri_attention.h -- C ABI of the B200 (sm_100a) TriAttention KV-compression round.
+ *
+ * One round, per (sequence, layer, KV head) "unit" holding N cached keys:
+ *   1. score every key with the offset-averaged trigonometric-series estimate plus the
+ *      concentration-weighted norm term, once per query head g of the GQA group, z-score
+ *      each head's scores over the unit's keys and take the max over g   (Sections 4.1-4.3);
+ *   2. keep the B keys with the highest final score                      (Section 4.3);
+ *   3. gather the kept K rows, V rows and positions into compacted slots, in slot order
+ *      (the eviction of Section 4.3: the cache physically shrinks to B rows).
+ *
+ * Conventions
+ *   - Every function returns a tri_status and never throws, traps or synchronises the device.
+ *   - "host" / "device" on a pointer says where the memory must live.  The caller owns every
+ *     buffer it passes, including the workspace; the library owns only tri_ctx.
+ *   - All launches go to the CUDA stream passed as `stream` (a cudaStream_t cast to void*,
+ *     NULL = the legacy default stream) and are asynchronous.  Errors the host can detect
+ *     (bad arguments, workspace too small) return before anything is launched.
+ *   - Units are indexed u = (layer * S + seq) * n_kv_heads + kv_head.  Per-unit outputs are
+ *     dense in u.  head_dim is 128 (64 frequency bands).
+ *   - Band layout (tri_model_desc.pair_layout): 0 pairs components (x[2f], x[2f+1]) as the
+ *     rotation matrix of Section 2.1 is written; 1 pairs (x[f], x[f+64]).
+ */
+#ifndef TRI_ATTENTION_H
+#define TRI_ATTENTION_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TRI_OK = 0,
+    TRI_ERR_INVALID_ARG = 1,   /* NULL where a pointer is required, bad size or stride         */
+    TRI_ERR_UNSUPPORTED = 2,   /* head_dim != 128, group_size > 16, page_size % 16 != 0, ...    */
+    TRI_ERR_WORKSPACE = 3,     /* ws_bytes < tri_workspace_bytes(...)                           */
+    TRI_ERR_CUDA = 4,          /* a CUDA runtime call failed; see tri_last_cuda_error()         */
+    TRI_ERR_DEVICE_CHECK = 5   /* (reported through *device_status, never returned)             */
+} tri_status;
+
+/* Model and method constants.  Host memory; copied by tri_create. */
+typedef struct {
+    int32_t n_layers;          /* L                                                            */
+    int32_t n_kv_heads;        /* H                                                            */
+    int32_t group_size;        /* G query heads per KV head (1..16); query head = kv_head*G+g  */
+    int32_t head_dim;          /* must be 128                                                  */
+    double  rope_theta;        /* RoPE base theta, omega_f = theta^(-2f/d)      (Section 2.1)  */
+    int32_t pair_layout;       /* 0 interleaved, 1 half-split                                  */
+    int32_t n_offsets;         /* |D|, 1..64                                                   */
+    const int64_t *offsets;    /* host [n_offsets]; the future offsets D of Section 4.2
+                                  (the paper's set is {1, 2, 4, ..., 2^16}); values >= 0        */
+    int32_t norm_variant;      /* weight of |k_f| in the norm term:
+                                  0: E|q_f| - |E q_f|   (Section 4.2, default)
+                                  1: E|q_f|             (S_norm^(0) of Section 4.1)
+                                  2: none (trigonometric term only)                            */
+} tri_model_desc;
+
+typedef struct tri_ctx tri_ctx;
+
+/*
+ * Builds the per-model context on the current CUDA device: device copies of the calibration
+ * statistics of Section 4.1 and the offset-averaged phasors (1/|D|) sum_delta e^{i omega_f delta}.
+ *   q_center     host [L][H*G][128] fp32  E[q_f]: pre-RoPE query centre, in the band layout above
+ *   q_mean_norm  host [L][H*G][64]  fp32  E|q_f|
+ * Allocates device memory (the only entry point besides tri_destroy that touches the allocator).
+ */
+tri_status tri_create(const tri_model_desc *desc, const float *q_center, const float *q_mean_norm,
+                      tri_ctx **out);
+tri_status tri_destroy(tri_ctx *ctx);
+
+/*
+ * A view of a K/V cache.  All pointers are device pointers owned by the caller.  Strides are in
+ * ELEMENTS of the respective array and must be multiples of 8 (16-byte rows); the innermost
+ * (head_dim) stride is 1.
+ *
+ * contiguous (paged == 0):  row(l, s, h, n) at  l*stride_layer + s*stride_seq + h*stride_head + n*stride_tok
+ * paged      (paged == 1):  page = page_table[s*max_pages_per_seq + n / page_size],
+ *                           row at  l*stride_layer + page*stride_page + h*stride_head + (n % page_size)*stride_slot
+ */
+typedef struct {
+    void *k;                   /* keys: bf16 post-RoPE (k_kind 0) or fp32 pre-RoPE (k_kind 1)   */
+    void *v;                   /* values, bf16, same strides as k; NULL = no value cache        */
+    int32_t k_kind;            /* 0: bf16 as cached by the model (post-RoPE) -- the fast path
+                                  1: fp32 pre-RoPE vectors (needs `positions` or slot = position) */
+    int32_t paged;
+    int64_t stride_layer, stride_seq, stride_head, stride_tok;
+    const int32_t *page_table; /* device [S][max_pages_per_seq]                                  */
+    int32_t max_pages_per_seq;
+    int32_t page_size;         /* multiple of 16                                                 */
+    int32_t n_pages;           /* pages in the pool: ids outside [0, n_pages) are reported through
+                                  device_status and their rows skipped; 0 = ids are not checked   */
+    int64_t stride_page, stride_slot;
+    const int32_t *seq_lens;   /* device [S]: keys currently cached per sequence (source views)  */
+    int32_t *positions;        /* device [L][S][H][n_max] original RoPE position per slot, or
+                                  NULL meaning position == slot index                           */
+    int32_t n_max;             /* row capacity per unit (>= every seq_lens[s])                   */
+} tri_cache_view;
+
+/* Bytes of device workspace any of the calls below needs for (S sequences, n_max, budget). */
+size_t tri_workspace_bytes(const tri_ctx *ctx, int32_t S, int32_t n_max, int32_t budget);
+
+/*
+ * Scoring (Sections 4.1-4.3).  For every unit and key n < seq_lens[s]:
+ *   raw[g]   = (1/|D|) sum_{delta in D} S_trig^(g)(k, p_q - p_k + delta) + S_norm^(g)(k)
+ *   scores   = max_g (raw[g] - mu_g) / sigma_g,  mu_g, sigma_g over the unit's keys (population
+ *              standard deviation; a head with sigma_g = 0 contributes 0).
+ *   cur_pos  device [S] int64: p_q, the position of the next query of each sequence
+ *   scores   device [U][n_max] fp32 (entries >= seq_lens[s] are not written)
+ *   raw      device [U][n_max][G] fp32 or NULL: if given, also receives the un-normalised scores
+ *   ws       device workspace, 256-byte aligned
+ * V is never read.
+ */
+tri_status tri_score(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                     float *scores, float *raw, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Top-B retention (Section 4.3).  Per unit keeps the `budget` highest scores among the first
+ * seq_lens[s] entries; equal scores: the lower slot wins; seq_lens[s] <= budget keeps all.
+ *   scores    device [U][n_max] fp32 (finite values)
+ *   kept_idx  device [U][budget] int32: kept slots in ascending order (entries >= count untouched)
+ *   kept_cnt  device [U] int32: min(budget, seq_lens[s])
+ */
+tri_status tri_select(tri_ctx *ctx, const float *scores, const int32_t *seq_lens, int32_t S,
+                      int32_t n_max, int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
+                      void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Eviction as an order-preserving gather (Section 4.3):  dst row j <- src row kept_idx[j] for K, V
+ * and positions, j < kept_cnt[u].  dst may alias src (same k pointer and strides): the in-place
+ * schedule then moves rows tile by tile in ascending order inside one thread block per unit.
+ * dst->seq_lens is ignored; new_seq_lens (device [S], may be NULL) receives kept_cnt of the
+ * sequence.  If dst->positions is given it receives the positions of the kept rows.
+ */
+tri_status tri_compact(tri_ctx *ctx, const tri_cache_view *src, const int32_t *kept_idx,
+                       const int32_t *kept_cnt, int32_t S, int32_t budget, const tri_cache_view *dst,
+                       int32_t *new_seq_lens, void *stream);
+
+/*
+ * The fused round: score, select, compact, in one call (a handful of launches, no host sync).
+ *   kept_idx, kept_cnt   device outputs as in tri_select, or NULL to use workspace
+ *   device_status        device int32[1] or NULL; set to TRI_ERR_DEVICE_CHECK if a kernel met a
+ *                        page id outside [0, n_pages) -- such rows are skipped, never dereferenced
+ */
+tri_status tri_compress(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                        int32_t budget, const tri_cache_view *dst, int32_t *kept_idx,
+                        int32_t *kept_cnt, int32_t *new_seq_lens, int32_t *device_status,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The fused round for a cache that lives in HOST memory (contiguous views only): copies K, V
+ * (and positions) of src to the device staging view, runs tri_compress, and copies the
+ * compacted rows, positions and counts back, all on `stream`.
+ *   src_host / dst_host  views whose k, v, positions, seq_lens pointers are (pinned) host memory
+ *   src_dev  / dst_dev   device views of identical shape used as staging (caller-allocated)
+ *   cur_pos_host         host [S] int64;  cur_pos_dev device [S] staging
+ *   kept_cnt_host        host [U] int32 output
+ */
+tri_status tri_compress_host(tri_ctx *ctx, const tri_cache_view *src_host, const tri_cache_view *src_dev,
+                             int32_t S, const int64_t *cur_pos_host, int64_t *cur_pos_dev, int32_t budget,
+                             const tri_cache_view *dst_host, const tri_cache_view *dst_dev,
+                             int32_t *kept_cnt_host, int32_t *kept_cnt_dev,
+                             void *ws, size_t ws_bytes, void *stream);
+
+/* Number of kernel launches one tri_compress call issues for this shape (for launch accounting). */
+int32_t tri_compress_launches(const tri_ctx *ctx, const tri_cache_view *src, const tri_cache_view *dst);
+
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char *tri_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRI_ATTENTION_H */

@@ -1,0 +1,414 @@
+// Host side of the C ABI declared in include/tri_attention.h: argument checks, workspace carving and
+// kernel launches.  Nothing here synchronises the device or allocates after tri_create.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "tri_compact.cuh"
+#include "tri_score.cuh"
+#include "tri_select.cuh"
+
+using namespace tri;
+
+struct tri_ctx {
+    tri_model_desc desc;
+    int device;
+    double *omega_d;     // [64]
+    double2 *dbar_d;     // [64]  (1/|D|) sum_delta e^{i omega_f delta}
+    float *qc_d;         // [L][H*G][128]
+    float *mw_d;         // [L][H*G][64]   weight of |k_f| in the norm term
+};
+
+static thread_local char g_err[256] = "";
+
+static tri_status cuda_fail(cudaError_t e, const char *what)
+{
+    snprintf(g_err, sizeof g_err, "%s: %s", what, cudaGetErrorString(e));
+    return TRI_ERR_CUDA;
+}
+#define TRI_CUDA(call)                                            \
+    do {                                                          \
+        cudaError_t e_ = (call);                                  \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call);       \
+    } while (0)
+
+extern "C" const char *tri_last_cuda_error(void) { return g_err; }
+
+// ----------------------------------------------------------------------------------------------
+// context
+// ----------------------------------------------------------------------------------------------
+extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_center, const float *q_mean_norm,
+                                 tri_ctx **out)
+{
+    if (!desc || !q_center || !q_mean_norm || !out) return TRI_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (desc->n_layers <= 0 || desc->n_kv_heads <= 0 || desc->group_size <= 0 || !(desc->rope_theta > 0.0))
+        return TRI_ERR_INVALID_ARG;
+    if (desc->n_offsets <= 0 || desc->n_offsets > 64 || !desc->offsets) return TRI_ERR_INVALID_ARG;
+    for (int i = 0; i < desc->n_offsets; ++i)
+        if (desc->offsets[i] < 0) return TRI_ERR_INVALID_ARG;
+    if (desc->pair_layout < 0 || desc->pair_layout > 1 || desc->norm_variant < 0 || desc->norm_variant > 2)
+        return TRI_ERR_INVALID_ARG;
+    if (desc->head_dim != kHeadDim || desc->group_size > kMaxGroup) return TRI_ERR_UNSUPPORTED;
+
+    tri_ctx *c = new (std::nothrow) tri_ctx();
+    if (!c) return TRI_ERR_INVALID_ARG;
+    c->desc = *desc;
+    c->desc.offsets = nullptr;
+    c->omega_d = nullptr; c->dbar_d = nullptr; c->qc_d = nullptr; c->mw_d = nullptr;
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaGetDevice"); }
+
+    // omega_f = theta^(-2f/d) (Section 2.1) and the offset-averaged phasor of Section 4.2, in double
+    double omega[kBands];
+    double2 dbar[kBands];
+    for (int f = 0; f < kBands; ++f) {
+        omega[f] = std::exp(-(2.0 * f / kHeadDim) * std::log(desc->rope_theta));
+        double re = 0.0, im = 0.0;
+        for (int i = 0; i < desc->n_offsets; ++i) {
+            double a = omega[f] * (double)desc->offsets[i];
+            re += std::cos(a);
+            im += std::sin(a);
+        }
+        dbar[f] = make_double2(re / desc->n_offsets, im / desc->n_offsets);
+    }
+    const size_t nq = (size_t)desc->n_layers * desc->n_kv_heads * desc->group_size;
+    std::vector<float> mw(nq * kBands);
+    for (size_t i = 0; i < nq; ++i)
+        for (int f = 0; f < kBands; ++f) {
+            int ir = desc->pair_layout == 0 ? 2 * f : f, ii = desc->pair_layout == 0 ? 2 * f + 1 : f + kBands;
+            double cr = q_center[i * kHeadDim + ir], ci = q_center[i * kHeadDim + ii];
+            double en = q_mean_norm[i * kBands + f];
+            double w = desc->norm_variant == 0 ? en - std::sqrt(cr * cr + ci * ci)
+                     : desc->norm_variant == 1 ? en : 0.0;
+            mw[i * kBands + f] = (float)w;
+        }
+    tri_status st = TRI_OK;
+    do {
+        if ((e = cudaMalloc(&c->omega_d, sizeof omega)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&c->dbar_d, sizeof dbar)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&c->qc_d, nq * kHeadDim * sizeof(float))) != cudaSuccess) break;
+        if ((e = cudaMalloc(&c->mw_d, nq * kBands * sizeof(float))) != cudaSuccess) break;
+        if ((e = cudaMemcpy(c->omega_d, omega, sizeof omega, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(c->dbar_d, dbar, sizeof dbar, cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(c->qc_d, q_center, nq * kHeadDim * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(c->mw_d, mw.data(), nq * kBands * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
+    } while (0);
+    if (e != cudaSuccess) {
+        st = cuda_fail(e, "tri_create");
+        tri_destroy(c);
+        return st;
+    }
+    *out = c;
+    return TRI_OK;
+}
+
+extern "C" tri_status tri_destroy(tri_ctx *c)
+{
+    if (!c) return TRI_OK;
+    cudaFree(c->omega_d);
+    cudaFree(c->dbar_d);
+    cudaFree(c->qc_d);
+    cudaFree(c->mw_d);
+    delete c;
+    return TRI_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// workspace
+// ----------------------------------------------------------------------------------------------
+namespace {
+
+struct Plan {
+    int32_t U, chunk, nchunks;
+    size_t off_E, off_raw, off_part, off_scores, off_idx, off_cnt, total;
+};
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Keys per scoring block: about 96 warp tiles (1,536 keys), evened out over the unit.
+void pick_chunk(int32_t n_max, int32_t *chunk, int32_t *nchunks)
+{
+    int32_t tiles = (n_max + kTileKeys - 1) / kTileKeys;
+    int32_t nch = (tiles + 48) / 96;
+    if (nch < 1) nch = 1;
+    int32_t per = (tiles + nch - 1) / nch;
+    *chunk = per * kTileKeys;
+    *nchunks = (tiles + per - 1) / per;
+}
+
+Plan make_plan(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget)
+{
+    Plan p;
+    const int G = c->desc.group_size;
+    p.U = c->desc.n_layers * S * c->desc.n_kv_heads;
+    pick_chunk(n_max, &p.chunk, &p.nchunks);
+    size_t o = 0;
+    p.off_E = o;      o += align256((size_t)S * kBands * sizeof(double2));
+    p.off_raw = o;    o += align256((size_t)p.U * n_max * G * sizeof(float));
+    p.off_part = o;   o += align256((size_t)p.U * p.nchunks * G * sizeof(double2));
+    p.off_scores = o; o += align256((size_t)p.U * n_max * sizeof(float));
+    p.off_idx = o;    o += align256((size_t)p.U * (size_t)(budget > 0 ? budget : 0) * sizeof(int32_t));
+    p.off_cnt = o;    o += align256((size_t)p.U * sizeof(int32_t));
+    p.total = o;
+    return p;
+}
+
+View to_view(const tri_cache_view *v)
+{
+    View w;
+    w.k = (char *)v->k; w.v = (char *)v->v;
+    w.k_kind = v->k_kind; w.paged = v->paged;
+    w.stride_layer = v->stride_layer; w.stride_seq = v->stride_seq;
+    w.stride_head = v->stride_head; w.stride_tok = v->stride_tok;
+    w.page_table = v->page_table; w.max_pages_per_seq = v->max_pages_per_seq;
+    w.page_size = v->page_size; w.n_pages = v->n_pages;
+    w.stride_page = v->stride_page; w.stride_slot = v->stride_slot;
+    w.seq_lens = v->seq_lens; w.positions = v->positions; w.n_max = v->n_max;
+    return w;
+}
+
+tri_status check_view(const tri_cache_view *v, bool need_lens)
+{
+    if (!v || !v->k) return TRI_ERR_INVALID_ARG;
+    if (v->k_kind < 0 || v->k_kind > 1 || v->n_max <= 0) return TRI_ERR_INVALID_ARG;
+    if (need_lens && !v->seq_lens) return TRI_ERR_INVALID_ARG;
+    if (((uintptr_t)v->k & 15) || ((uintptr_t)v->v & 15)) return TRI_ERR_INVALID_ARG;
+    if (v->stride_layer % 8 || v->stride_head % 8) return TRI_ERR_INVALID_ARG;
+    if (v->paged) {
+        if (!v->page_table || v->max_pages_per_seq <= 0 || v->page_size <= 0) return TRI_ERR_INVALID_ARG;
+        if (v->page_size % kTileKeys) return TRI_ERR_UNSUPPORTED;
+        if (v->stride_page % 8 || v->stride_slot % 8 || v->stride_slot < kHeadDim) return TRI_ERR_INVALID_ARG;
+        if ((int64_t)v->max_pages_per_seq * v->page_size < v->n_max) return TRI_ERR_INVALID_ARG;
+    } else {
+        if (v->stride_seq % 8 || v->stride_tok % 8 || v->stride_tok < kHeadDim) return TRI_ERR_INVALID_ARG;
+    }
+    return TRI_OK;
+}
+
+tri_status check_launch(const char *what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, what);
+    return TRI_OK;
+}
+
+template <int LAYOUT>
+void launch_score_bf16(int NT, dim3 grid, cudaStream_t st, const ScoreParams &sp)
+{
+    if (NT == 1) k_score_bf16<1, LAYOUT><<<grid, kScoreThreads, 0, st>>>(sp);
+    else if (NT == 2) k_score_bf16<2, LAYOUT><<<grid, kScoreThreads, 0, st>>>(sp);
+    else k_score_bf16<4, LAYOUT><<<grid, kScoreThreads, 0, st>>>(sp);
+}
+
+// fold -> raw scores -> z-score/max.  3 launches.
+tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, float *scores,
+                     float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st)
+{
+    const int G = c->desc.group_size;
+    double2 *E = (double2 *)(ws + pl.off_E);
+    float *raw = raw_out ? raw_out : (float *)(ws + pl.off_raw);
+    double2 *part = (double2 *)(ws + pl.off_part);
+
+    k_fold_phasors<<<S, kBands, 0, st>>>(c->omega_d, c->dbar_d, cur_pos, E);
+    tri_status r = check_launch("k_fold_phasors");
+    if (r != TRI_OK) return r;
+
+    ScoreParams sp;
+    sp.src = to_view(src);
+    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G;
+    sp.chunk = pl.chunk; sp.nchunks = pl.nchunks;
+    sp.E = E; sp.qc = c->qc_d; sp.mw = c->mw_d;
+    sp.raw = raw; sp.partials = part; sp.device_status = device_status;
+    dim3 grid((unsigned)((size_t)pl.U * pl.nchunks));
+    if (src->k_kind == 0) {
+        int NT = G <= 4 ? 1 : (G <= 8 ? 2 : 4);
+        if (c->desc.pair_layout == 0) launch_score_bf16<0>(NT, grid, st, sp);
+        else launch_score_bf16<1>(NT, grid, st, sp);
+    } else {
+        if (c->desc.pair_layout == 0)
+            k_score_f32_pre<0><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);
+        else
+            k_score_f32_pre<1><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);
+    }
+    if ((r = check_launch("k_score")) != TRI_OK) return r;
+
+    NormParams np;
+    np.raw = raw; np.partials = part; np.seq_lens = src->seq_lens; np.scores = scores;
+    np.S = S; np.H = c->desc.n_kv_heads; np.G = G; np.n_max = src->n_max;
+    np.chunk = pl.chunk; np.nchunks = pl.nchunks;
+    k_normalize<<<grid, 256, 0, st>>>(np);
+    return check_launch("k_normalize");
+}
+
+tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
+                      int32_t budget, int32_t *kept_idx, int32_t *kept_cnt, int32_t *new_seq_lens,
+                      int32_t U, cudaStream_t st)
+{
+    SelectParams p;
+    p.scores = scores; p.seq_lens = seq_lens; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
+    p.new_seq_lens = new_seq_lens;
+    p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget;
+    k_select<<<U, kSelThreads, 0, st>>>(p);
+    return check_launch("k_select");
+}
+
+bool aliases(const tri_cache_view *a, const tri_cache_view *b)
+{
+    return a->k == b->k || (a->v && a->v == b->v) || (a->positions && a->positions == b->positions);
+}
+
+tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx, const int32_t *kept_cnt,
+                       int32_t S, int32_t budget, const tri_cache_view *dst, int32_t *new_seq_lens,
+                       int32_t *device_status, int32_t U, cudaStream_t st)
+{
+    CompactParams p;
+    p.src = to_view(src); p.dst = to_view(dst);
+    p.kept_idx = kept_idx; p.kept_cnt = kept_cnt; p.new_seq_lens = new_seq_lens;
+    p.S = S; p.H = c->desc.n_kv_heads; p.budget = budget;
+    p.k_esize = src->k_kind == 0 ? 2 : 4;
+    p.k_vec = kHeadDim * p.k_esize / 16;
+    p.v_vec = (src->v && dst->v) ? kHeadDim * 2 / 16 : 0;
+    p.device_status = device_status;
+    if (aliases(src, dst)) {
+        k_compact_inplace<<<U, kInplaceThreads, 0, st>>>(p);
+    } else {
+        dim3 grid(U, (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock);
+        k_gather<<<grid, kGatherThreads, 0, st>>>(p);
+    }
+    return check_launch("k_compact");
+}
+
+tri_status check_common(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget)
+{
+    if (!c || S <= 0 || n_max <= 0 || budget <= 0) return TRI_ERR_INVALID_ARG;
+    int64_t U = (int64_t)c->desc.n_layers * S * c->desc.n_kv_heads;
+    if (U > (1 << 24) || (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock > 65535) return TRI_ERR_UNSUPPORTED;
+    return TRI_OK;
+}
+
+}  // namespace
+
+extern "C" size_t tri_workspace_bytes(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget)
+{
+    if (!c || S <= 0 || n_max <= 0) return 0;
+    return make_plan(c, S, n_max, budget).total;
+}
+
+// ----------------------------------------------------------------------------------------------
+// entry points
+// ----------------------------------------------------------------------------------------------
+extern "C" tri_status tri_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                float *scores, float *raw, void *ws, size_t ws_bytes, void *stream)
+{
+    tri_status r;
+    if (!c || !src || !cur_pos || !scores || !ws) return TRI_ERR_INVALID_ARG;
+    if ((r = check_view(src, true)) != TRI_OK) return r;
+    if ((r = check_common(c, S, src->n_max, 1)) != TRI_OK) return r;
+    if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
+    Plan pl = make_plan(c, S, src->n_max, 0);
+    if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
+    return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream);
+}
+
+extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S,
+                                 int32_t n_max, int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
+                                 void *ws, size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;   // the selection keeps its histograms in shared memory
+    tri_status r;
+    if (!c || !scores || !seq_lens || !kept_idx || !kept_cnt) return TRI_ERR_INVALID_ARG;
+    if ((r = check_common(c, S, n_max, budget)) != TRI_OK) return r;
+    int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
+    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, nullptr, U, (cudaStream_t)stream);
+}
+
+extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx,
+                                  const int32_t *kept_cnt, int32_t S, int32_t budget, const tri_cache_view *dst,
+                                  int32_t *new_seq_lens, void *stream)
+{
+    tri_status r;
+    if (!c || !kept_idx || !kept_cnt) return TRI_ERR_INVALID_ARG;
+    if ((r = check_view(src, false)) != TRI_OK) return r;
+    if ((r = check_view(dst, false)) != TRI_OK) return r;
+    if ((r = check_common(c, S, src->n_max, budget)) != TRI_OK) return r;
+    if (dst->n_max < budget && dst->n_max < src->n_max) return TRI_ERR_INVALID_ARG;
+    if (src->k_kind != dst->k_kind) return TRI_ERR_INVALID_ARG;
+    int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
+    return run_compact(c, src, kept_idx, kept_cnt, S, budget, dst, new_seq_lens, nullptr, U, (cudaStream_t)stream);
+}
+
+extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                   int32_t budget, const tri_cache_view *dst, int32_t *kept_idx,
+                                   int32_t *kept_cnt, int32_t *new_seq_lens, int32_t *device_status,
+                                   void *ws, size_t ws_bytes, void *stream)
+{
+    tri_status r;
+    if (!c || !cur_pos || !ws) return TRI_ERR_INVALID_ARG;
+    if ((r = check_view(src, true)) != TRI_OK) return r;
+    if ((r = check_view(dst, false)) != TRI_OK) return r;
+    if ((r = check_common(c, S, src->n_max, budget)) != TRI_OK) return r;
+    if (dst->n_max < budget && dst->n_max < src->n_max) return TRI_ERR_INVALID_ARG;
+    if (src->k_kind != dst->k_kind) return TRI_ERR_INVALID_ARG;
+    if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
+    Plan pl = make_plan(c, S, src->n_max, budget);
+    if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *w = (char *)ws;
+    float *scores = (float *)(w + pl.off_scores);
+    int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
+    int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
+    if ((r = run_score(c, src, S, cur_pos, scores, nullptr, w, pl, device_status, st)) != TRI_OK) return r;
+    if ((r = run_select(c, scores, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, st)) != TRI_OK)
+        return r;
+    return run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, pl.U, st);
+}
+
+extern "C" int32_t tri_compress_launches(const tri_ctx *c, const tri_cache_view *src, const tri_cache_view *dst)
+{
+    (void)c; (void)src; (void)dst;
+    return 5;   // fold, score, normalise, select, gather
+}
+
+extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_host, const tri_cache_view *src_dev,
+                                        int32_t S, const int64_t *cur_pos_host, int64_t *cur_pos_dev, int32_t budget,
+                                        const tri_cache_view *dst_host, const tri_cache_view *dst_dev,
+                                        int32_t *kept_cnt_host, int32_t *kept_cnt_dev,
+                                        void *ws, size_t ws_bytes, void *stream)
+{
+    if (!c || !src_host || !src_dev || !dst_host || !dst_dev || !cur_pos_host || !cur_pos_dev || !kept_cnt_dev)
+        return TRI_ERR_INVALID_ARG;
+    if (src_host->paged || src_dev->paged || dst_host->paged || dst_dev->paged) return TRI_ERR_UNSUPPORTED;
+    if (src_host->stride_layer != src_dev->stride_layer || dst_host->stride_layer != dst_dev->stride_layer ||
+        src_host->n_max != src_dev->n_max || dst_host->n_max != dst_dev->n_max)
+        return TRI_ERR_INVALID_ARG;
+    if (!src_host->seq_lens || !src_dev->seq_lens || !src_host->k || !dst_host->k) return TRI_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int L = c->desc.n_layers, H = c->desc.n_kv_heads;
+    const size_t kes = src_host->k_kind == 0 ? 2 : 4;
+    const size_t src_elems = (size_t)L * src_host->stride_layer, dst_elems = (size_t)L * dst_host->stride_layer;
+    const size_t U = (size_t)L * S * H;
+    TRI_CUDA(cudaMemcpyAsync(src_dev->k, src_host->k, src_elems * kes, cudaMemcpyHostToDevice, st));
+    if (src_host->v && src_dev->v)
+        TRI_CUDA(cudaMemcpyAsync(src_dev->v, src_host->v, src_elems * 2, cudaMemcpyHostToDevice, st));
+    if (src_host->positions && src_dev->positions)
+        TRI_CUDA(cudaMemcpyAsync(src_dev->positions, src_host->positions, U * src_host->n_max * sizeof(int32_t),
+                                 cudaMemcpyHostToDevice, st));
+    TRI_CUDA(cudaMemcpyAsync((void *)src_dev->seq_lens, src_host->seq_lens, S * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, st));
+    TRI_CUDA(cudaMemcpyAsync(cur_pos_dev, cur_pos_host, S * sizeof(int64_t), cudaMemcpyHostToDevice, st));
+    tri_status r = tri_compress(c, src_dev, S, cur_pos_dev, budget, dst_dev, nullptr, kept_cnt_dev, nullptr, nullptr,
+                                ws, ws_bytes, stream);
+    if (r != TRI_OK) return r;
+    TRI_CUDA(cudaMemcpyAsync(dst_host->k, dst_dev->k, dst_elems * kes, cudaMemcpyDeviceToHost, st));
+    if (dst_host->v && dst_dev->v)
+        TRI_CUDA(cudaMemcpyAsync(dst_host->v, dst_dev->v, dst_elems * 2, cudaMemcpyDeviceToHost, st));
+    if (dst_host->positions && dst_dev->positions)
+        TRI_CUDA(cudaMemcpyAsync(dst_host->positions, dst_dev->positions, U * dst_host->n_max * sizeof(int32_t),
+                                 cudaMemcpyDeviceToHost, st));
+    if (kept_cnt_host)
+        TRI_CUDA(cudaMemcpyAsync(kept_cnt_host, kept_cnt_dev, U * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    return TRI_OK;
+}

@@ -1,0 +1,308 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 CPU oracle on the same
+seeded inputs.  Sizes are chosen so that the oracle finishes in seconds while every unit still spans
+several scoring blocks and a ragged tail."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_04921_b200 import binding as tb
+from paper_2604_04921_b200 import workloads as W
+
+from parity import (check_compacted, check_kept, check_scores, check_unit, make_ctx, oracle_unit, run_compress,
+                    src_view, unit_index)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _all_units(w):
+    return [(l, s, h) for l in range(w.k.shape[0]) for s in range(w.spec.n_seqs) for h in range(w.spec.n_kv_heads)]
+
+
+def test_config0_tiny_bf16_post_rope():
+    w = W.make_workload(W.SPECS["tiny"], DEV)
+    B = w.spec.budget
+    ref = oracle_unit(w, 0, 0, 0, B)
+    res = run_compress(w, B)
+    st = check_unit(w, res, ref, 0, 0, 0, B)
+    assert int(res["status"].item()) == 0
+    assert int(res["new_seq_lens"][0].item()) == B
+    assert st["raw_err"] < 0.1      # far inside the tolerance: errors are ~1e-5 relative
+
+
+def test_config0_tiny_fp32_pre_rope():
+    """The configuration's own input format: fp32 pre-RoPE keys, position = slot."""
+    w = W.make_workload(W.SPECS["tiny"], DEV)
+    sp, B = w.spec, w.spec.budget
+    kpre = w.k_pre_fp32
+    N = sp.n_keys
+    qc = w.q_center[0].double().numpy()
+    qn = w.q_mean_norm[0].double().numpy()
+    raw_o = oracle.score_raw(kpre[0, 0, 0].double().cpu().numpy(), np.arange(N), N, qc, qn, theta=sp.theta)
+    _, s_o = oracle.normalize(raw_o)
+    idx_o = oracle.select(s_o, B)
+    ctx = make_ctx(w)
+    src = tb.CacheView(kpre, None, seq_lens=w.seq_lens)
+    ws = ctx.workspace(1, N, B)
+    scores = torch.empty(1, N, dtype=torch.float32, device=DEV)
+    raw = torch.empty(1, N, 1, dtype=torch.float32, device=DEV)
+    ctx.score(src, w.cur_pos, scores, ws, raw=raw)
+    ref = dict(raw=raw_o, s_final=s_o, idx=idx_o)
+    check_scores(raw[0].cpu().numpy(), scores[0].cpu().numpy(), ref)
+    kout = torch.zeros(1, 1, 1, B, 128, dtype=torch.float32, device=DEV)
+    kept_idx = torch.empty(1, B, dtype=torch.int32, device=DEV)
+    kept_cnt = torch.empty(1, dtype=torch.int32, device=DEV)
+    ctx.compress(src, w.cur_pos, B, tb.CacheView(kout, None), ws, kept_idx=kept_idx, kept_cnt=kept_cnt)
+    torch.cuda.synchronize()
+    check_kept(kept_idx[0].cpu().numpy(), int(kept_cnt[0]), ref, B)
+    sel = kept_idx[0].long()
+    assert torch.equal(kout[0, 0, 0], kpre[0, 0, 0][sel])
+
+
+def test_config1_shape_scaled():
+    """Qwen3-8B head geometry (G = 4), 2 layers x 2 KV heads, 5,000 keys: 3 scoring blocks + ragged tail."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(n_layers=2, n_kv_heads=2, n_keys=5000, budget=300)
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget)
+    assert int(res["status"].item()) == 0
+    for (l, s, h) in _all_units(w):
+        check_unit(w, res, oracle_unit(w, l, s, h, sp.budget), l, s, h, sp.budget)
+
+
+def test_config2_shape_steady_state():
+    """Batch of sequences holding budget + 128 keys at scattered original positions."""
+    sp = W.SPECS["qwen3_8b_steady_b64"].scaled(n_layers=1, n_kv_heads=2, n_seqs=3)
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget)
+    assert res["new_seq_lens"].tolist() == [sp.budget] * 3
+    for (l, s, h) in _all_units(w):
+        check_unit(w, res, oracle_unit(w, l, s, h, sp.budget), l, s, h, sp.budget)
+
+
+def test_config3_shape_mixed_noise():
+    """Per-head noise std in [0.2, 1.0]: concentrated and diffuse heads in one launch."""
+    sp = W.SPECS["qwen3_8b_long_128k"].scaled(n_layers=1, n_kv_heads=3, n_keys=12345, budget=1000)
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget)
+    for (l, s, h) in _all_units(w):
+        check_unit(w, res, oracle_unit(w, l, s, h, sp.budget), l, s, h, sp.budget)
+
+
+@pytest.mark.parametrize("in_place", [False, True])
+def test_config4_shape_ragged_paged(in_place):
+    """G = 8, ragged lengths, 16-token pages in a shuffled table; compacted rows go back into pages."""
+    sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(n_layers=2, n_kv_heads=2, n_seqs=3, n_keys=2500, n_keys_min=300,
+                                                  budget=512)
+    w = W.make_workload(sp, DEV)
+    refs = {u: oracle_unit(w, *u, sp.budget) for u in _all_units(w)}      # before any in-place write
+    res = run_compress(w, sp.budget, in_place=in_place)
+    assert int(res["status"].item()) == 0
+    lens = w.seq_lens.tolist()
+    assert res["new_seq_lens"].tolist() == [min(n, sp.budget) for n in lens]
+    for u, ref in refs.items():
+        check_unit(w, res, ref, *u, sp.budget)
+
+
+def test_in_place_contiguous_matches_out_of_place():
+    sp = W.SPECS["qwen3_8b_steady_b64"].scaled(n_layers=1, n_kv_heads=2, n_seqs=2)
+    w = W.make_workload(sp, DEV)
+    a = run_compress(w, sp.budget, want_scores=False)
+    k0, v0, p0 = w.k.clone(), w.v.clone(), w.positions.clone()
+    b = run_compress(w, sp.budget, in_place=True, want_scores=False)
+    assert torch.equal(a["kept_idx"], b["kept_idx"])
+    B = sp.budget
+    assert torch.equal(a["k_out"].view(torch.int16), w.k[:, :, :, :B].view(torch.int16))
+    assert torch.equal(a["v_out"].view(torch.int16), w.v[:, :, :, :B].view(torch.int16))
+    assert torch.equal(a["pos_out"], w.positions[:, :, :, :B])
+    # rows beyond the budget are untouched
+    assert torch.equal(k0[:, :, :, B:].view(torch.int16), w.k[:, :, :, B:].view(torch.int16))
+    assert torch.equal(p0[:, :, :, B:], w.positions[:, :, :, B:])
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 5, 8, 16])
+def test_group_sizes(G):
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name=f"g{G}", n_layers=1, n_kv_heads=2, group_size=G, n_keys=1111,
+                                                budget=100)
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget)
+    for (l, s, h) in _all_units(w):
+        check_unit(w, res, oracle_unit(w, l, s, h, sp.budget), l, s, h, sp.budget)
+
+
+@pytest.mark.parametrize("norm_variant", [1, 2])
+def test_norm_variants(norm_variant):
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="nv", n_layers=1, n_kv_heads=1, n_keys=2000, budget=128)
+    w = W.make_workload(sp, DEV)
+    ctx = make_ctx(w, norm_variant=norm_variant)
+    res = run_compress(w, sp.budget, ctx=ctx)
+    check_unit(w, res, oracle_unit(w, 0, 0, 0, sp.budget, norm_variant=norm_variant), 0, 0, 0, sp.budget)
+
+
+def test_other_offset_sets():
+    """The offset ablation's sets are runtime parameters (Appendix on future offsets)."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="off", n_layers=1, n_kv_heads=1, n_keys=1500, budget=64)
+    w = W.make_workload(sp, DEV)
+    for offs in ([1], [1, 2, 4, 8, 16, 32, 64, 128], list(range(1, 65537, 4096)) + [65536]):
+        ctx = make_ctx(w, offsets=offs)
+        res = run_compress(w, sp.budget, ctx=ctx)
+        check_unit(w, res, oracle_unit(w, 0, 0, 0, sp.budget, offsets=offs), 0, 0, 0, sp.budget)
+
+
+def test_half_split_layout():
+    """pair_layout 1: band f = (x[f], x[f+64]).  Same data permuted must give the same result."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="hs", n_layers=1, n_kv_heads=2, n_keys=1800, budget=200)
+    w = W.make_workload(sp, DEV)
+    perm = torch.cat([torch.arange(0, 128, 2), torch.arange(1, 128, 2)])
+    res0 = run_compress(w, sp.budget)
+    w2 = W.Workload(sp, w.q_center[..., perm].contiguous(), w.q_mean_norm, w.k[..., perm.to(DEV)].contiguous(),
+                    w.v, w.seq_lens, w.cur_pos, None, None)
+    ctx = make_ctx(w2, pair_layout=1)
+    res1 = run_compress(w2, sp.budget, ctx=ctx)
+    assert torch.equal(res0["kept_idx"], res1["kept_idx"])
+    assert torch.allclose(res0["raw"], res1["raw"], rtol=0, atol=2e-4)
+    for (l, s, h) in _all_units(w2):
+        kk, vv, pos = w2.unit_rows(l, s, h)
+        G = sp.group_size
+        raw, sfin, idx = oracle.unit_bf16(W.bf16_bits(kk), pos.numpy(), int(w2.cur_pos[s]),
+                                          w2.q_center[l, h * G:(h + 1) * G].double().numpy(),
+                                          w2.q_mean_norm[l, h * G:(h + 1) * G].double().numpy(), sp.budget, layout=1)
+        check_unit(w2, res1, dict(raw=raw, s_final=sfin, idx=idx, k=kk, v=vv, pos=pos), l, s, h, sp.budget)
+
+
+def test_degenerate_sizes():
+    """N <= B keeps everything in order; N = 1; B = 1; a sequence of length 0 beside a full one."""
+    base = W.SPECS["qwen3_8b_oneshot_32k"]
+    for n, B in [(100, 512), (512, 512), (1, 4), (700, 1), (17, 16)]:
+        sp = base.scaled(name=f"deg{n}_{B}", n_layers=1, n_kv_heads=2, n_keys=n, budget=B)
+        w = W.make_workload(sp, DEV)
+        res = run_compress(w, B)
+        for (l, s, h) in _all_units(w):
+            check_unit(w, res, oracle_unit(w, l, s, h, B), l, s, h, B)
+        if n <= B:
+            u = res["kept_idx"][:, :n].cpu()
+            assert torch.equal(u, torch.arange(n, dtype=torch.int32).expand_as(u))
+    # ragged batch with an empty sequence
+    sp = base.scaled(name="empty", n_layers=1, n_kv_heads=1, n_seqs=3, n_keys=600, budget=64)
+    w = W.make_workload(sp, DEV)
+    w.seq_lens = torch.tensor([600, 0, 37], dtype=torch.int32, device=DEV)
+    w.cur_pos = torch.tensor([600, 0, 37], dtype=torch.int64, device=DEV)
+    res = run_compress(w, 64)
+    assert res["kept_cnt"].tolist() == [64, 0, 37]
+    assert res["new_seq_lens"].tolist() == [64, 0, 37]
+    for s in (0, 2):
+        check_unit(w, res, oracle_unit(w, 0, s, 0, 64), 0, s, 0, 64)
+    assert torch.all(res["k_out"][0, 1] == 0)
+
+
+def test_constant_head_contributes_zero():
+    """A query head with zero centre and E|q_f| = 0 scores every key 0: sigma = 0, z = 0 for that head."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="const", n_layers=1, n_kv_heads=1, group_size=2, n_keys=900,
+                                                budget=90)
+    w = W.make_workload(sp, DEV)
+    w.q_center[0, 1] = 0
+    w.q_mean_norm[0, 1] = 0
+    res = run_compress(w, sp.budget)
+    ref = oracle_unit(w, 0, 0, 0, sp.budget)
+    assert np.all(ref["raw"][1] == 0)
+    check_unit(w, res, ref, 0, 0, 0, sp.budget)
+    assert float(res["scores"][0, :900].min()) >= 0.0
+
+
+def test_select_bit_exact_with_ties():
+    """tri_select alone on fp32 scores full of ties: indices must equal the oracle's exactly."""
+    g = torch.Generator().manual_seed(5)
+    cases = [(1, 5000, 777, 50), (3, 131072, 4096, 0), (4, 9999, 9998, 7), (2, 4096, 1, 3), (2, 70000, 35000, 1000)]
+    for U, n, B, levels in cases:
+        x = torch.randn(U, n, generator=g)
+        if levels:
+            x = torch.round(x * levels / 6) / levels          # many exactly equal values
+        x[0, : min(n, 10)] = 0.0
+        sc = x.to(DEV)
+        lens = torch.tensor([n], dtype=torch.int32, device=DEV)
+        ctx = tb.TriContext(U, 1, 1, torch.zeros(U, 1, 128), torch.zeros(U, 1, 64))
+        idx = torch.full((U, B), -1, dtype=torch.int32, device=DEV)
+        cnt = torch.zeros(U, dtype=torch.int32, device=DEV)
+        ctx.select(sc, lens, n, B, idx, cnt)
+        torch.cuda.synchronize()
+        assert cnt.tolist() == [min(B, n)] * U
+        for u in range(U):
+            want = oracle.select(x[u].double().numpy(), B)
+            assert np.array_equal(idx[u].cpu().numpy(), want), (U, n, B, levels, u)
+    # negative values, -0.0 vs +0.0 and infinities keep the float order
+    x = torch.tensor([[0.0, -0.0, -1.0, float("inf"), 1e-40, -1e-40, 3.0, float("-inf")]])
+    ctx = tb.TriContext(1, 1, 1, torch.zeros(1, 1, 128), torch.zeros(1, 1, 64))
+    idx = torch.full((1, 3), -1, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ctx.select(x.to(DEV), torch.tensor([8], dtype=torch.int32, device=DEV), 8, 3, idx, cnt)
+    assert sorted(idx[0].tolist()) == [3, 4, 6]
+
+
+def test_compact_standalone_and_rerun_determinism():
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="det", n_layers=2, n_kv_heads=2, n_keys=4000, budget=256)
+    w = W.make_workload(sp, DEV)
+    a = run_compress(w, sp.budget)
+    b = run_compress(w, sp.budget)
+    for key in ("scores", "raw", "kept_idx", "kept_cnt"):
+        assert torch.equal(a[key], b[key]), key
+    assert torch.equal(a["k_out"].view(torch.int16), b["k_out"].view(torch.int16))
+    # tri_compact on its own from the kept indices reproduces the fused call's rows
+    ctx = a["ctx"]
+    k2, v2 = torch.zeros_like(a["k_out"]), torch.zeros_like(a["v_out"])
+    p2 = torch.zeros_like(a["pos_out"])
+    lens = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ctx.compact(src_view(w), a["kept_idx"], a["kept_cnt"], 1, sp.budget, tb.CacheView(k2, v2, positions=p2), lens)
+    torch.cuda.synchronize()
+    assert torch.equal(k2.view(torch.int16), a["k_out"].view(torch.int16))
+    assert torch.equal(v2.view(torch.int16), a["v_out"].view(torch.int16))
+    assert torch.equal(p2, a["pos_out"]) and lens.tolist() == [sp.budget]
+
+
+def test_bad_page_id_sets_status_not_fault():
+    """A page id outside the pool is reported through device_status; its rows are skipped."""
+    sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name="badpage", n_layers=1, n_kv_heads=1, n_seqs=2, n_keys=400,
+                                                  n_keys_min=200, budget=64)
+    w = W.make_workload(sp, DEV)
+    w.page_table[0, 3] = 10 ** 6
+    res = run_compress(w, sp.budget, want_scores=False)
+    assert int(res["status"].item()) == 5
+
+
+def test_host_errors_launch_nothing():
+    w = W.make_workload(W.SPECS["tiny"].scaled(n_keys=256, budget=32), DEV)
+    ctx = make_ctx(w)
+    src = src_view(w)
+    ws = ctx.workspace(1, 256, 32)
+    dst = tb.CacheView(torch.zeros(1, 1, 1, 32, 128, dtype=torch.bfloat16, device=DEV), None)
+    with pytest.raises(tb.TriError) as e:
+        ctx.compress(src, w.cur_pos, 32, dst, ws[:1024])
+    assert e.value.code == 3
+    with pytest.raises(tb.TriError) as e:
+        ctx.compress(src, w.cur_pos, 0, dst, ws)
+    assert e.value.code == 1
+    small = tb.CacheView(torch.zeros(1, 1, 1, 8, 128, dtype=torch.bfloat16, device=DEV), None)
+    with pytest.raises(tb.TriError) as e:
+        ctx.compress(src, w.cur_pos, 32, small, ws)
+    assert e.value.code == 1
+    torch.cuda.synchronize()
+
+
+def test_full_size_config1_sampled_units():
+    """The benchmark's own workload and launch configuration (36 x 8 units of 32,768 keys, B = 2,048):
+    whole-job invariants plus the oracle on two sampled units."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"]
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget, want_scores=False)
+    assert int(res["status"].item()) == 0
+    assert torch.all(res["kept_cnt"] == sp.budget)
+    idx = res["kept_idx"]
+    assert torch.all(idx[:, 1:] > idx[:, :-1]) and int(idx.min()) >= 0 and int(idx.max()) < sp.n_keys
+    # every compacted row is a bit copy of the row its index names
+    L, H = sp.n_layers, sp.n_kv_heads
+    gi = idx.view(L, 1, H, sp.budget, 1).long().expand(L, 1, H, sp.budget, 128)
+    assert torch.equal(torch.gather(w.k, 3, gi).view(torch.int16), res["k_out"].view(torch.int16))
+    assert torch.equal(torch.gather(w.v, 3, gi).view(torch.int16), res["v_out"].view(torch.int16))
+    assert torch.equal(res["pos_out"].view(-1, sp.budget), idx)
+    for (l, h) in [(0, 0), (35, 7)]:
+        ref = oracle_unit(w, l, 0, h, sp.budget)
+        check_unit(w, res, ref, l, 0, h, sp.budget)
