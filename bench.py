@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the fused compression round (tri_compress) on synthetic Qwen3-shaped caches.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole hot path (phasor fold, scoring, z-score/max, top-B select, gather
+compaction) over every (sequence, layer, KV head) unit of the workload.  Prints ONE JSON line.
+
+* value      keys scored+selected+compacted per second, inputs resident in HBM, CUDA events around K
+             steps, max over ranks (N > 1: independent replicas, one per GPU, "weak" scaling).
+* e2e        the same metric through tri_compress_host: pinned host K/V in, compacted K/V out, copies
+             inside the timed region.
+* roofline   the scoring kernel (it streams the whole key cache): algorithmic bytes / its mean launch
+             time, measured with CUDA events recorded by the library between its launches in a second
+             pass of K steps.
+* cpu_baseline  the float64 oracle, as it stands, on a bounded sample of units of the same workload.
+
+--impl reference times that oracle alone (rank 0 only), one sampled unit per step.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tri_compress keys scored+selected+compacted per sec"
+UNIT = "keys/s"
+DEFAULT_WORKLOAD = "qwen3_8b_oneshot_32k"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for nm, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(seq_lens, units_per_seq, budget):
+    """256 N (stream K) + 1036 min(B, N) (re-read kept K, read kept V, write both, idx + positions)."""
+    tot = 0
+    for n in seq_lens:
+        tot += units_per_seq * (256 * n + 1036 * min(budget, n))
+    return tot
+
+
+def oracle_sample(spec, units, budget):
+    """Time the CPU oracle on the given (layer, seq, head) units.  Returns (keys, seconds)."""
+    import oracle
+    from paper_2604_04921_b200 import workloads as W
+    keys, secs, cache = 0, 0.0, {}
+    for (l, s, h) in units:
+        if l not in cache:
+            cache.clear()
+            cache[l] = W.make_workload(spec, "cpu", layer0=l, n_layers=1)
+        w = cache[l]
+        kk, vv, pos = w.unit_rows(0, s, h)
+        G = spec.group_size
+        bits = W.bf16_bits(kk)
+        qc = w.q_center[0, h * G:(h + 1) * G].double().numpy()
+        qn = w.q_mean_norm[0, h * G:(h + 1) * G].double().numpy()
+        t0 = time.perf_counter()
+        raw, sfin, idx = oracle.unit_bf16(bits, pos.numpy(), int(w.cur_pos[s]), qc, qn, budget, theta=spec.theta)
+        oracle.compact(W.bf16_bits(kk), idx)
+        oracle.compact(W.bf16_bits(vv), idx)
+        secs += time.perf_counter() - t0
+        keys += kk.shape[0]
+    return keys, secs
+
+
+def sample_units(spec, count):
+    """Deterministic spread of units: first/last layer and head first, then striding through."""
+    L, S, H = spec.n_layers, spec.n_seqs, spec.n_kv_heads
+    out = [(0, 0, 0), (L - 1, S - 1, H - 1)]
+    i = 1
+    while len(out) < count:
+        u = (i * 7919) % (L * S * H)
+        out.append((u // (S * H), (u // H) % S, u % H))
+        i += 1
+    return out[:count]
+
+
+def run_reference(args, spec):
+    """--impl reference: the oracle as it stands, one sampled unit per step, on the host cores."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    oracle.build()
+    units = sample_units(spec, args.warmup + args.steps)
+    oracle_sample(spec, units[:max(1, min(args.warmup, 1))], spec.budget)     # warm-up: page in, build
+    keys, secs = oracle_sample(spec, units[args.warmup:args.warmup + args.steps], spec.budget)
+    val = keys / secs
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": spec.name, "units_per_step": 1, "keys_per_unit": spec.n_keys,
+                       "budget": spec.budget},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": f"{args.steps} units of {spec.n_keys} keys (one per step) out of "
+                                       f"{spec.n_layers * spec.n_seqs * spec.n_kv_heads}"},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (a slab); 0 = all")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+
+    from paper_2604_04921_b200 import workloads as W
+    spec = W.SPECS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, spec)
+        return
+
+    import torch
+    from paper_2604_04921_b200 import binding as tb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression round has no CPU implementation")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    tb.lib()   # fails loudly if the CUDA library has not been built
+
+    L = args.layers if args.layers > 0 else spec.n_layers
+    w = W.make_workload(spec, dev, layer0=0, n_layers=L)
+    S, H, G, B = spec.n_seqs, spec.n_kv_heads, spec.group_size, spec.budget
+    ctx = tb.TriContext(L, H, G, w.q_center, w.q_mean_norm, rope_theta=spec.theta)
+    src = tb.CacheView(w.k, w.v, seq_lens=w.seq_lens, positions=w.positions, page_table=w.page_table)
+    n_max = src.c_view().n_max
+    U = L * S * H
+    if w.paged:
+        # compacted rows are written back into the sequence's own pages (in place)
+        dst = tb.CacheView(w.k, w.v, page_table=w.page_table, n_max=n_max)
+    else:
+        k2 = torch.empty(L, S, H, B, 128, dtype=torch.bfloat16, device=dev)
+        v2 = torch.empty_like(k2)
+        p2 = torch.empty(L, S, H, B, dtype=torch.int32, device=dev)
+        dst = tb.CacheView(k2, v2, positions=p2)
+    ws = ctx.workspace(S, n_max, B, dev)
+    kept_cnt = torch.zeros(U, dtype=torch.int32, device=dev)
+    lens = w.seq_lens.tolist()
+    keys_per_step = sum(lens) * L * H
+    abytes = algorithmic_bytes(lens, L * H, B)
+    launches_per_step = ctx.compress_launches(src, dst)
+
+    def step():
+        ctx.compress(src, w.cur_pos, B, dst, ws, kept_cnt=kept_cnt)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+
+    # per-kernel durations: second pass, events recorded by the library between its launches
+    ctx.profile_begin()
+    per = {k: 0.0 for k in ctx.KERNELS}
+    for _ in range(args.steps):
+        step()
+        for k, v in ctx.profile_read().items():
+            per[k] += v / args.steps
+    ctx.profile_end()
+    clocks = sampler.stop() if rank == 0 else None
+
+    peak, peak_src = measured_peaks()
+    score_bytes = 256 * keys_per_step
+    score_gbs = score_bytes / (per["score"] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": world * keys_per_step / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": spec.name + (f"[first {L} layers]" if L != spec.n_layers else ""),
+                   "units": U, "layers": L, "kv_heads": H, "group_size": G, "seqs": S, "keys_per_step": keys_per_step,
+                   "budget": B, "storage_dtype": "bf16", "paged": bool(w.paged),
+                   "compaction": "in place into the sequence's pages" if w.paged else "out of place",
+                   "l2": f"inputs larger than L2: {(w.k.numel() + w.v.numel()) * 2 / 1e9:.2f} GB of K+V read per step",
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "hbm": {"algorithmic_bytes_per_step": abytes, "achieved_gbs": abytes / (ms_step * 1e-3) / 1e9,
+                "frac_of_measured_copy_peak": abytes / (ms_step * 1e-3) / 1e9 / peak,
+                "frac_of_nominal_8tbs": abytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+        "roofline": {"kernel": "k_score_bf16", "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": score_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"]},
+        "kernel_ms": per,
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clocks,
+    }
+
+    # ---- end to end through tri_compress_host: pinned host buffers, copies inside the timed region ----
+    if not args.no_e2e and not w.paged:
+        e2e_steps = max(2, min(args.steps, 5))
+        hk = torch.empty(w.k.shape, dtype=w.k.dtype, pin_memory=True).copy_(w.k)
+        hv = torch.empty(w.v.shape, dtype=w.v.dtype, pin_memory=True).copy_(w.v)
+        hpos = None if w.positions is None else torch.empty(w.positions.shape, dtype=torch.int32, pin_memory=True).copy_(w.positions)
+        hlens = torch.empty(S, dtype=torch.int32, pin_memory=True).copy_(w.seq_lens)
+        hcur = torch.empty(S, dtype=torch.int64, pin_memory=True).copy_(w.cur_pos)
+        hk2 = torch.empty(k2.shape, dtype=k2.dtype, pin_memory=True)
+        hv2 = torch.empty(k2.shape, dtype=k2.dtype, pin_memory=True)
+        hp2 = torch.empty(p2.shape, dtype=torch.int32, pin_memory=True)
+        hcnt = torch.empty(U, dtype=torch.int32, pin_memory=True)
+        dlens = torch.empty_like(w.seq_lens)
+        dcur = torch.empty_like(w.cur_pos)
+        src_h = tb.CacheView(hk, hv, seq_lens=hlens, positions=hpos)
+        src_d = tb.CacheView(w.k, w.v, seq_lens=dlens, positions=w.positions)
+        dst_h = tb.CacheView(hk2, hv2, positions=hp2)
+
+        def step_host():
+            ctx.compress_host(src_h, src_d, hcur, dcur, B, dst_h, dst, hcnt, kept_cnt, ws)
+
+        step_host()
+        barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            step_host()
+        e1.record()
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item()) / e2e_steps
+        assert int(hcnt.min()) == min(B, min(lens))
+        h2d = (hk.numel() + hv.numel()) * 2 + (0 if hpos is None else hpos.numel() * 4) + S * 12
+        d2h = (hk2.numel() + hv2.numel()) * 2 + hp2.numel() * 4 + U * 4
+        line["e2e"] = {"value": world * keys_per_step / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+                       "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "call": "tri_compress_host (pinned host K/V/positions in, compacted K/V/positions/counts out)"}
+        del hk, hv, hk2, hv2
+    else:
+        line["e2e"] = None
+
+    # ---- the oracle on this machine's host cores, bounded sample (rank 0, N = 1 only) ----
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        t0 = time.perf_counter()
+        units = sample_units(spec.scaled(n_layers=L), 64)
+        keys = secs = 0.0
+        used = 0
+        for uidx in units:
+            k_, s_ = oracle_sample(spec, [uidx], B)
+            keys += k_; secs += s_; used += 1
+            if time.perf_counter() - t0 > 15.0:
+                break
+        line["cpu_baseline"] = {"value": keys / secs, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": f"{used} of {U} units ({int(keys)} keys), oracle time {secs:.1f} s"}
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

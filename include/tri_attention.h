@@ -166,6 +166,17 @@ tri_status tri_compress_host(tri_ctx *ctx, const tri_cache_view *src_host, const
 /* Number of kernel launches one tri_compress call issues for this shape (for launch accounting). */
 int32_t tri_compress_launches(const tri_ctx *ctx, const tri_cache_view *src, const tri_cache_view *dst);
 
+/*
+ * Measurement aid (the paper has no counterpart): between tri_profile_begin and tri_profile_end every
+ * tri_compress call records a CUDA event before and after each of its 5 kernels (phasor fold, raw
+ * scoring, z-score/max, top-B select, gather) on its stream.  tri_profile_read waits for the last
+ * call's final event and writes the 5 kernel durations in milliseconds to ms[0..4] (host).
+ * tri_profile_begin creates the events; it is the only one of the three that allocates.
+ */
+tri_status tri_profile_begin(tri_ctx *ctx);
+tri_status tri_profile_read(tri_ctx *ctx, float *ms);
+tri_status tri_profile_end(tri_ctx *ctx);
+
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char *tri_last_cuda_error(void);
 

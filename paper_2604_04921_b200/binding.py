@@ -23,7 +23,8 @@ HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cu
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",
-           "tri_compress", "tri_compress_host", "tri_compress_launches", "tri_last_cuda_error"]
+           "tri_compress", "tri_compress_host", "tri_compress_launches", "tri_last_cuda_error",
+           "tri_profile_begin", "tri_profile_read", "tri_profile_end"]
 
 STATUS = {0: "TRI_OK", 1: "TRI_ERR_INVALID_ARG", 2: "TRI_ERR_UNSUPPORTED", 3: "TRI_ERR_WORKSPACE",
           4: "TRI_ERR_CUDA", 5: "TRI_ERR_DEVICE_CHECK"}
@@ -101,6 +102,11 @@ def lib():
     L.tri_compress_host.restype = ctypes.c_int
     L.tri_compress_launches.argtypes = [P, VP, VP]
     L.tri_compress_launches.restype = i32
+    for fn in (L.tri_profile_begin, L.tri_profile_end):
+        fn.argtypes = [P]
+        fn.restype = ctypes.c_int
+    L.tri_profile_read.argtypes = [P, P]
+    L.tri_profile_read.restype = ctypes.c_int
     L.tri_last_cuda_error.argtypes = []
     L.tri_last_cuda_error.restype = ctypes.c_char_p
     _lib = L
@@ -261,6 +267,20 @@ class TriContext:
                                        _ptr(cur_pos_dev), budget, ctypes.byref(c), ctypes.byref(d),
                                        _ptr(kept_cnt_host), _ptr(kept_cnt_dev), _ptr(ws), ws.numel(), _stream()),
                "tri_compress_host")
+
+    KERNELS = ("fold_phasors", "score", "normalize", "select", "compact")
+
+    def profile_begin(self):
+        _check(lib().tri_profile_begin(self._h), "tri_profile_begin")
+
+    def profile_read(self):
+        """Durations (ms) of the 5 kernels of the last compress() call; waits for that call."""
+        ms = (ctypes.c_float * 5)()
+        _check(lib().tri_profile_read(self._h, ctypes.cast(ms, ctypes.c_void_p)), "tri_profile_read")
+        return dict(zip(self.KERNELS, [float(x) for x in ms]))
+
+    def profile_end(self):
+        _check(lib().tri_profile_end(self._h), "tri_profile_end")
 
     def compress_launches(self, src: CacheView, dst: CacheView) -> int:
         a, b = src.c_view(), dst.c_view()

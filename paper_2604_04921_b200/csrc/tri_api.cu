@@ -12,6 +12,8 @@
 
 using namespace tri;
 
+constexpr int kProfEvents = 6;   // boundaries of the 5 launches of tri_compress
+
 struct tri_ctx {
     tri_model_desc desc;
     int device;
@@ -19,7 +21,15 @@ struct tri_ctx {
     double2 *dbar_d;     // [64]  (1/|D|) sum_delta e^{i omega_f delta}
     float *qc_d;         // [L][H*G][128]
     float *mw_d;         // [L][H*G][64]   weight of |k_f| in the norm term
+    bool profiling;      // tri_profile_begin .. tri_profile_end: time each kernel of tri_compress
+    cudaEvent_t ev[kProfEvents];
 };
+
+// Records event i on the stream while profiling is on (between the launches of tri_compress).
+static void mark(tri_ctx *c, int i, cudaStream_t st)
+{
+    if (c->profiling) cudaEventRecord(c->ev[i], st);
+}
 
 static thread_local char g_err[256] = "";
 
@@ -58,6 +68,7 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
     c->desc = *desc;
     c->desc.offsets = nullptr;
     c->omega_d = nullptr; c->dbar_d = nullptr; c->qc_d = nullptr; c->mw_d = nullptr;
+    c->profiling = false;
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaGetDevice"); }
 
@@ -108,6 +119,7 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
 extern "C" tri_status tri_destroy(tri_ctx *c)
 {
     if (!c) return TRI_OK;
+    if (c->profiling) for (int i = 0; i < kProfEvents; ++i) cudaEventDestroy(c->ev[i]);
     cudaFree(c->omega_d);
     cudaFree(c->dbar_d);
     cudaFree(c->qc_d);
@@ -212,9 +224,11 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     float *raw = raw_out ? raw_out : (float *)(ws + pl.off_raw);
     double2 *part = (double2 *)(ws + pl.off_part);
 
+    mark(c, 0, st);
     k_fold_phasors<<<S, kBands, 0, st>>>(c->omega_d, c->dbar_d, cur_pos, E);
     tri_status r = check_launch("k_fold_phasors");
     if (r != TRI_OK) return r;
+    mark(c, 1, st);
 
     ScoreParams sp;
     sp.src = to_view(src);
@@ -234,13 +248,16 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
             k_score_f32_pre<1><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);
     }
     if ((r = check_launch("k_score")) != TRI_OK) return r;
+    mark(c, 2, st);
 
     NormParams np;
     np.raw = raw; np.partials = part; np.seq_lens = src->seq_lens; np.scores = scores;
     np.S = S; np.H = c->desc.n_kv_heads; np.G = G; np.n_max = src->n_max;
     np.chunk = pl.chunk; np.nchunks = pl.nchunks;
     k_normalize<<<grid, 256, 0, st>>>(np);
-    return check_launch("k_normalize");
+    r = check_launch("k_normalize");
+    mark(c, 3, st);
+    return r;
 }
 
 tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
@@ -252,7 +269,9 @@ tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, 
     p.new_seq_lens = new_seq_lens;
     p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget;
     k_select<<<U, kSelThreads, 0, st>>>(p);
-    return check_launch("k_select");
+    tri_status r = check_launch("k_select");
+    mark(c, 4, st);
+    return r;
 }
 
 bool aliases(const tri_cache_view *a, const tri_cache_view *b)
@@ -278,7 +297,9 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
         dim3 grid(U, (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock);
         k_gather<<<grid, kGatherThreads, 0, st>>>(p);
     }
-    return check_launch("k_compact");
+    tri_status r = check_launch("k_compact");
+    mark(c, 5, st);
+    return r;
 }
 
 tri_status check_common(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget)
@@ -410,5 +431,39 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
                                  cudaMemcpyDeviceToHost, st));
     if (kept_cnt_host)
         TRI_CUDA(cudaMemcpyAsync(kept_cnt_host, kept_cnt_dev, U * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    return TRI_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// per-kernel timing of tri_compress (measurement aid)
+// ----------------------------------------------------------------------------------------------
+extern "C" tri_status tri_profile_begin(tri_ctx *c)
+{
+    if (!c) return TRI_ERR_INVALID_ARG;
+    if (c->profiling) return TRI_OK;
+    for (int i = 0; i < kProfEvents; ++i) {
+        cudaError_t e = cudaEventCreate(&c->ev[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(c->ev[j]);
+            return cuda_fail(e, "cudaEventCreate");
+        }
+    }
+    c->profiling = true;
+    return TRI_OK;
+}
+
+extern "C" tri_status tri_profile_read(tri_ctx *c, float *ms)
+{
+    if (!c || !ms || !c->profiling) return TRI_ERR_INVALID_ARG;
+    TRI_CUDA(cudaEventSynchronize(c->ev[kProfEvents - 1]));
+    for (int i = 0; i + 1 < kProfEvents; ++i) TRI_CUDA(cudaEventElapsedTime(&ms[i], c->ev[i], c->ev[i + 1]));
+    return TRI_OK;
+}
+
+extern "C" tri_status tri_profile_end(tri_ctx *c)
+{
+    if (!c) return TRI_ERR_INVALID_ARG;
+    if (c->profiling) for (int i = 0; i < kProfEvents; ++i) cudaEventDestroy(c->ev[i]);
+    c->profiling = false;
     return TRI_OK;
 }
