@@ -54,18 +54,63 @@ __device__ __forceinline__ void mma_tf32_1688(float (&d)[4], uint32_t a0, uint32
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint32_t to_tf32(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;\n" : "=r"(r) : "f"(x));
-    return r;
-}
-
 __device__ __forceinline__ float fast_sqrt(float x)
 {
     float r;
     asm("sqrt.approx.ftz.f32 %0, %1;\n" : "=f"(r) : "f"(x));
     return r;
+}
+
+// Upper part of an fp32 that is exactly representable in tf32 (10 explicit mantissa bits).  With
+// lo = x - hi (exact), hi + lo carries x to ~2^-22 through two tf32 MMAs.
+__device__ __forceinline__ uint32_t to_tf32(float x) { return __float_as_uint(x) & 0xffffe000u; }
+
+// Packed fp32 pairs (sm_100 f32x2 arithmetic): two lanes per instruction.
+__device__ __forceinline__ uint64_t pack2(float a, float b)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &a, float &b)
+{
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;\n" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;\n" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// Magnitudes of two bands held as bf16 (re, im) pairs in xa and xb, split for tf32:
+// hi = (hi_a, hi_b) as tf32 bit patterns, lo = the exact remainders.
+__device__ __forceinline__ void band_mags2(uint32_t xa, uint32_t xb, uint32_t &hi_a, uint32_t &hi_b,
+                                           uint32_t &lo_a, uint32_t &lo_b)
+{
+    uint64_t re = pack2(__uint_as_float(xa << 16), __uint_as_float(xb << 16));
+    uint64_t im = pack2(__uint_as_float(xa & 0xffff0000u), __uint_as_float(xb & 0xffff0000u));
+    float sa, sb;
+    unpack2(fma2(re, re, mul2(im, im)), sa, sb);
+    float ma = fast_sqrt(sa), mb = fast_sqrt(sb);
+    hi_a = to_tf32(ma);
+    hi_b = to_tf32(mb);
+    float la, lb;
+    unpack2(sub2(pack2(ma, mb), pack2(__uint_as_float(hi_a), __uint_as_float(hi_b))), la, lb);
+    lo_a = __float_as_uint(la);
+    lo_b = __float_as_uint(lb);
 }
 
 // 16-byte streaming load of cache rows: read once, keep out of L1.
@@ -239,22 +284,12 @@ k_score_bf16(const ScoreParams p)
             for (int j = 0; j < 4; ++j) {
                 const uint32_t *x0 = reinterpret_cast<const uint32_t *>(&A0[j]);
                 const uint32_t *x1 = reinterpret_cast<const uint32_t *>(&A1[j]);
-                float mg0[4], mg1[4];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    float re0 = __uint_as_float(x0[r] << 16), im0 = __uint_as_float(x0[r] & 0xffff0000u);
-                    float re1 = __uint_as_float(x1[r] << 16), im1 = __uint_as_float(x1[r] & 0xffff0000u);
-                    mg0[r] = fast_sqrt(fmaf(re0, re0, im0 * im0));
-                    mg1[r] = fast_sqrt(fmaf(re1, re1, im1 * im1));
-                }
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    uint32_t h00 = to_tf32(mg0[2 * e]), h10 = to_tf32(mg1[2 * e]);
-                    uint32_t h01 = to_tf32(mg0[2 * e + 1]), h11 = to_tf32(mg1[2 * e + 1]);
-                    uint32_t l00 = __float_as_uint(mg0[2 * e] - __uint_as_float(h00));
-                    uint32_t l10 = __float_as_uint(mg1[2 * e] - __uint_as_float(h10));
-                    uint32_t l01 = __float_as_uint(mg0[2 * e + 1] - __uint_as_float(h01));
-                    uint32_t l11 = __float_as_uint(mg1[2 * e + 1] - __uint_as_float(h11));
+                    // pair the same band of rows q and q+8: (a0, a1) and (a2, a3) are then born adjacent
+                    uint32_t h00, h01, l00, l01, h10, h11, l10, l11;
+                    band_mags2(x0[2 * e], x1[2 * e], h00, h10, l00, l10);           // k slot t
+                    band_mags2(x0[2 * e + 1], x1[2 * e + 1], h01, h11, l01, l11);   // k slot t+4
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         uint2 b = normB[nt][2 * j + e][lane];
