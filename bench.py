@@ -269,7 +269,7 @@ def main():
         "hbm": {"algorithmic_bytes_per_step": abytes, "achieved_gbs": abytes / (ms_step * 1e-3) / 1e9,
                 "frac_of_measured_copy_peak": abytes / (ms_step * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8tbs": abytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
-        "roofline": {"kernel": "k_score_bf16", "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": "k_score_tma", "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
                      "frac": score_gbs / peak, "traffic": None, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"]},
         "kernel_ms": per,

@@ -2,12 +2,14 @@
 // kernel launches.  Nothing here synchronises the device or allocates after tri_create.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
 
 #include "tri_compact.cuh"
 #include "tri_score.cuh"
+#include "tri_score_tma.cuh"
 #include "tri_select.cuh"
 
 using namespace tri;
@@ -207,12 +209,69 @@ tri_status check_launch(const char *what)
     return TRI_OK;
 }
 
-template <int LAYOUT>
-void launch_score_bf16(int NT, dim3 grid, cudaStream_t st, const ScoreParams &sp)
+// The key cache as a rank-5 bf16 tensor for the TMA unit: (dim, row, KV head, sequence | page, layer),
+// box = 64 dims x 16 rows, 128-byte swizzle.  Host-side encode only; nothing is allocated.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, CUtensorMap *out)
 {
-    if (NT == 1) k_score_bf16<1, LAYOUT><<<grid, kScoreThreads, 0, st>>>(sp);
-    else if (NT == 2) k_score_bf16<2, LAYOUT><<<grid, kScoreThreads, 0, st>>>(sp);
-    else k_score_bf16<4, LAYOUT><<<grid, kScoreThreads, 0, st>>>(sp);
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q);
+        if (e != cudaSuccess || !ptr) return cuda_fail(e == cudaSuccess ? cudaErrorUnknown : e, "cuTensorMapEncodeTiled lookup");
+        fn = (EncodeTiledFn)ptr;
+    }
+    auto bytes = [](int64_t elems) { return (cuuint64_t)(elems > 0 ? elems : 8) * 2; };
+    cuuint64_t dims[5], strides[4];
+    dims[0] = kHeadDim;
+    dims[2] = (cuuint64_t)c->desc.n_kv_heads;
+    dims[4] = (cuuint64_t)c->desc.n_layers;
+    if (v->paged) {
+        dims[1] = (cuuint64_t)v->page_size;
+        dims[3] = v->n_pages > 0 ? (cuuint64_t)v->n_pages : (cuuint64_t)0x7fffffff;
+        strides[0] = bytes(v->stride_slot);
+        strides[2] = bytes(v->stride_page);
+    } else {
+        dims[1] = (cuuint64_t)v->n_max;
+        dims[3] = (cuuint64_t)S;
+        strides[0] = bytes(v->stride_tok);
+        strides[2] = bytes(v->stride_seq);
+    }
+    strides[1] = bytes(v->stride_head);
+    strides[3] = bytes(v->stride_layer);
+    cuuint32_t box[5] = {kHeadDim / 2, kTileKeys, 1, 1, 1}, estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, v->k, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return TRI_ERR_CUDA;
+    }
+    return TRI_OK;
+}
+
+template <int NT, int LAYOUT>
+tri_status launch_score_tma_one(dim3 grid, cudaStream_t st, const CUtensorMap &map, const ScoreParams &sp)
+{
+    static bool configured = false;
+    if (!configured) {
+        TRI_CUDA(cudaFuncSetAttribute(k_score_tma<NT, LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreDynSmem));
+        configured = true;
+    }
+    k_score_tma<NT, LAYOUT><<<grid, kScoreThreads, kScoreDynSmem, st>>>(map, sp);
+    return TRI_OK;
+}
+
+template <int LAYOUT>
+tri_status launch_score_tma(int NT, dim3 grid, cudaStream_t st, const CUtensorMap &map, const ScoreParams &sp)
+{
+    if (NT == 1) return launch_score_tma_one<1, LAYOUT>(grid, st, map, sp);
+    if (NT == 2) return launch_score_tma_one<2, LAYOUT>(grid, st, map, sp);
+    return launch_score_tma_one<4, LAYOUT>(grid, st, map, sp);
 }
 
 // fold -> raw scores -> z-score/max.  3 launches.
@@ -239,8 +298,11 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     dim3 grid((unsigned)((size_t)pl.U * pl.nchunks));
     if (src->k_kind == 0) {
         int NT = G <= 4 ? 1 : (G <= 8 ? 2 : 4);
-        if (c->desc.pair_layout == 0) launch_score_bf16<0>(NT, grid, st, sp);
-        else launch_score_bf16<1>(NT, grid, st, sp);
+        CUtensorMap map;
+        if ((r = encode_key_map(c, src, S, &map)) != TRI_OK) return r;
+        r = c->desc.pair_layout == 0 ? launch_score_tma<0>(NT, grid, st, map, sp)
+                                     : launch_score_tma<1>(NT, grid, st, map, sp);
+        if (r != TRI_OK) return r;
     } else {
         if (c->desc.pair_layout == 0)
             k_score_f32_pre<0><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);

@@ -1,0 +1,302 @@
+// Raw scoring of bf16 post-RoPE keys: TMA -> swizzled shared memory -> ldmatrix -> tensor cores.
+//
+// Data movement.  The cache (contiguous or paged) is described to the TMA unit as a rank-5 bf16
+// tensor (dim, row-in-page-or-unit, KV head, sequence-or-page, layer).  Every warp runs its own
+// pipeline: for each of its 16-key tiles lane 0 issues two tiled bulk-tensor loads (left and right
+// 64-element halves of the 16 rows, 2 KB each, 128-byte swizzle) that complete on a per-(warp, stage)
+// mbarrier.  The warp waits (bounded), pulls the tile into registers with 8 ldmatrix.x4 -- which
+// yields the A fragments of mma.m16n8k16 directly -- and immediately re-arms the stage with the
+// tile kStages ahead, so the copy engine stays kStages tiles in front of the arithmetic.
+//
+// Arithmetic per k-step s (dims 16s..16s+15 of 16 keys):
+//   trig   one bf16 MMA of the fragment with the (hi, lo)-split W              (Sections 4.1, 4.2)
+//   norm   the fragment's four registers are four (re, im) pairs = four bands; their magnitudes,
+//          split hi + lo for tf32, are the A fragment of two m16n8k8 tf32 MMAs with m_f (Section 4.2)
+// both accumulate into the same fp32 accumulator: thread (q, t) ends with S~ of head 4nt + t for keys
+// q and q+8 of the tile.
+#pragma once
+#include <cuda.h>
+
+#include "tri_score.cuh"
+
+namespace tri {
+
+constexpr int kStages = 3;
+constexpr int kTileBytes = kTileKeys * kHeadDim * 2;                       // 4096
+constexpr int kScoreDynSmem = kScoreWarps * kStages * kTileBytes;          // 98304
+constexpr uint32_t kWaitPolls = 1u << 22;                                  // bound on every mbarrier wait
+constexpr int TRI_STATUS_TIMEOUT = 6;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Waits for the phase with the given parity; gives up after kWaitPolls polls and returns false.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < kWaitPolls; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, int c4)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];\n" ::"r"(dst),
+        "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr)
+                 : "memory");
+}
+
+// |(re_a, im_a)| and |(re_b, im_b)| split for tf32: hi as tf32 bit patterns, lo the exact remainders.
+__device__ __forceinline__ void mags2(float re_a, float im_a, float re_b, float im_b, uint32_t &hi_a,
+                                      uint32_t &hi_b, uint32_t &lo_a, uint32_t &lo_b)
+{
+    uint64_t re = pack2(re_a, re_b), im = pack2(im_a, im_b);
+    float sa, sb;
+    unpack2(fma2(re, re, mul2(im, im)), sa, sb);
+    float ma = fast_sqrt(sa), mb = fast_sqrt(sb);
+    hi_a = to_tf32(ma);
+    hi_b = to_tf32(mb);
+    float la, lb;
+    unpack2(sub2(pack2(ma, mb), pack2(__uint_as_float(hi_a), __uint_as_float(hi_b))), la, lb);
+    lo_a = __float_as_uint(la);
+    lo_b = __float_as_uint(lb);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
+template <int NT, int LAYOUT>
+__global__ void __launch_bounds__(kScoreThreads)
+k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
+{
+    extern __shared__ __align__(1024) uint8_t tiles[];   // [warp][stage][half][16 rows][128 B]
+    __shared__ float Wf[NT * 4][kHeadDim];
+    __shared__ float Mf[NT * 4][kBands];
+    __shared__ uint2 trigB[NT][8][32];
+    __shared__ uint2 normB[NT][8][32];
+    __shared__ double red[kScoreWarps][NT * 4][2];
+    __shared__ __align__(8) uint64_t bars[kScoreWarps][kStages];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int u = blockIdx.x / p.nchunks, chunk = blockIdx.x - u * p.nchunks;
+    const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
+    const int n = min(__ldg(p.src.seq_lens + s), p.src.n_max);
+    const int key_begin = chunk * p.chunk;
+    if (key_begin >= n) return;
+    const int key_end = min(key_begin + p.chunk, n);
+    const int G = p.G;
+    const int ntiles = (key_end - key_begin + kTileKeys - 1) / kTileKeys;
+    const int my_n = warp < ntiles ? (ntiles - warp + kScoreWarps - 1) / kScoreWarps : 0;
+
+    const uint32_t my_tiles = smem_u32(tiles) + warp * (kStages * kTileBytes);
+    const uint32_t my_bars = smem_u32(&bars[warp][0]);
+
+    // lane 0 of each warp arms stage `it % kStages` with tile `it` of this warp
+    auto issue = [&](int it) {
+        const int stage = it % kStages;
+        const int row = key_begin + (warp + kScoreWarps * it) * kTileKeys;
+        int c1 = row, c3 = s;
+        if (p.src.paged) {
+            const int pg = row / p.src.page_size;
+            int page = __ldg(p.src.page_table + (int64_t)s * p.src.max_pages_per_seq + pg);
+            if (p.src.n_pages > 0 && (page < 0 || page >= p.src.n_pages)) {
+                if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
+                page = 0;                          // stay inside the pool; the unit's output is unspecified
+            }
+            c1 = row - pg * p.src.page_size;
+            c3 = page;
+        }
+        const uint32_t bar = my_bars + stage * 8, dst = my_tiles + stage * kTileBytes;
+        mbar_expect_tx(bar, kTileBytes);
+        tma_load_5d(dst, &tmap, bar, 0, c1, h, c3, l);
+        tma_load_5d(dst + kTileBytes / 2, &tmap, bar, kHeadDim / 2, c1, h, c3, l);
+    };
+
+    if (lane == 0) {
+        for (int st = 0; st < kStages; ++st) mbar_init(my_bars + st * 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        for (int it = 0; it < kStages && it < my_n; ++it) issue(it);
+    }
+
+    // ---- fold, step 2 (overlaps the first loads): W_f^(g) = E[q_f]^(g) * E[s][f], split for the MMAs ----
+    for (int i = tid; i < NT * 4 * kBands; i += kScoreThreads) {
+        int g = i / kBands, f = i - g * kBands;
+        int ir = LAYOUT == 0 ? 2 * f : f, ii = LAYOUT == 0 ? 2 * f + 1 : f + kBands;
+        float wr = 0.f, wi = 0.f, m = 0.f;
+        if (g < G) {
+            const float *c = p.qc + ((int64_t)l * p.H * G + (int64_t)h * G + g) * kHeadDim;
+            double cr = c[ir], ci = c[ii];
+            double2 e = p.E[s * kBands + f];
+            wr = (float)(cr * e.x - ci * e.y);
+            wi = (float)(cr * e.y + ci * e.x);
+            m = p.mw[((int64_t)l * p.H * G + (int64_t)h * G + g) * kBands + f];
+        }
+        Wf[g][ir] = wr;
+        Wf[g][ii] = wi;
+        Mf[g][f] = m;
+    }
+    __syncthreads();
+    for (int i = tid; i < NT * 8 * 32; i += kScoreThreads) {
+        int ln = i & 31, st = (i >> 5) & 7, nt = i >> 8;
+        int col = ln >> 2, t = ln & 3;          // B fragment: column = lane/4, k slots from lane%4
+        int g = 4 * nt + (col >> 1), part = col & 1;
+        uint32_t w[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {            // k slots 2t, 2t+1, 2t+8, 2t+9 of step st
+            float v = Wf[g][16 * st + 2 * t + (x & 1) + 8 * (x >> 1)];
+            uint32_t hi = bf16_hi_bits(v);
+            w[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+        }
+        trigB[nt][st][ln] = make_uint2(w[0] | (w[1] << 16), w[2] | (w[3] << 16));
+        // norm: tf32 step st, k slot t and t+4
+        int b0, b1;
+        if (LAYOUT == 0) { b0 = 8 * st + t; b1 = 8 * st + 4 + t; }
+        else { int ss = st >> 1, hf = st & 1; b0 = 16 * ss + 2 * t + hf; b1 = 16 * ss + 8 + 2 * t + hf; }
+        float m0 = Mf[g][b0], m1 = Mf[g][b1];
+        uint32_t h0 = to_tf32(m0), h1 = to_tf32(m1);
+        normB[nt][st][ln] = part == 0 ? make_uint2(h0, h1)
+                                      : make_uint2(__float_as_uint(m0 - __uint_as_float(h0)),
+                                                   __float_as_uint(m1 - __uint_as_float(h1)));
+    }
+    __syncthreads();
+
+    const int q = lane >> 2, t = lane & 3;
+    float s1[NT], s2[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) { s1[nt] = 0.f; s2[nt] = 0.f; }
+    // ldmatrix source of this lane inside a tile: row lane%16, 16-byte chunk 2*(s%4) + lane/16 of half s/4,
+    // chunk index XORed with row%8 (128-byte swizzle)
+    const int lrow = lane & 15, lsel = lane >> 4;
+    float *rawu = p.raw + (int64_t)u * p.src.n_max * G;
+    bool timed_out = false;
+
+    for (int it = 0; it < my_n; ++it) {
+        const int stage = it % kStages;
+        const uint32_t bar = my_bars + stage * 8, base = my_tiles + stage * kTileBytes;
+        if (!mbar_wait_bounded(bar, (it / kStages) & 1)) { timed_out = true; break; }
+        uint32_t X[8][4];
+#pragma unroll
+        for (int st = 0; st < 8; ++st) {
+            const int c = 2 * (st & 3) + lsel;
+            ldmatrix_x4(X[st], base + (st >> 2) * (kTileBytes / 2) + lrow * 128 + ((c ^ (lrow & 7)) << 4));
+        }
+        __syncwarp();
+        if (lane == 0 && it + kStages < my_n) {
+            asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+            issue(it + kStages);
+        }
+
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+#pragma unroll
+        for (int st = 0; st < 8; ++st) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                uint2 b = trigB[nt][st][lane];
+                mma_bf16_16816(acc[nt], X[st][0], X[st][1], X[st][2], X[st][3], b.x, b.y);
+            }
+        }
+        if (LAYOUT == 0) {
+#pragma unroll
+            for (int st = 0; st < 8; ++st) {
+                uint32_t hA[4], lA[4];
+                mags2(bf16_lo(X[st][0]), bf16_hi(X[st][0]), bf16_lo(X[st][1]), bf16_hi(X[st][1]), hA[0], hA[1], lA[0], lA[1]);
+                mags2(bf16_lo(X[st][2]), bf16_hi(X[st][2]), bf16_lo(X[st][3]), bf16_hi(X[st][3]), hA[2], hA[3], lA[2], lA[3]);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    uint2 b = normB[nt][st][lane];
+                    mma_tf32_1688(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
+                    mma_tf32_1688(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int ss = 0; ss < 4; ++ss) {
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    uint32_t hA[4], lA[4];
+                    const uint32_t *re = X[ss], *im = X[ss + 4];
+                    if (hf == 0) {
+                        mags2(bf16_lo(re[0]), bf16_lo(im[0]), bf16_lo(re[1]), bf16_lo(im[1]), hA[0], hA[1], lA[0], lA[1]);
+                        mags2(bf16_lo(re[2]), bf16_lo(im[2]), bf16_lo(re[3]), bf16_lo(im[3]), hA[2], hA[3], lA[2], lA[3]);
+                    } else {
+                        mags2(bf16_hi(re[0]), bf16_hi(im[0]), bf16_hi(re[1]), bf16_hi(im[1]), hA[0], hA[1], lA[0], lA[1]);
+                        mags2(bf16_hi(re[2]), bf16_hi(im[2]), bf16_hi(re[3]), bf16_hi(im[3]), hA[2], hA[3], lA[2], lA[3]);
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        uint2 b = normB[nt][2 * ss + hf][lane];
+                        mma_tf32_1688(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
+                        mma_tf32_1688(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
+                    }
+                }
+            }
+        }
+
+        // columns (2t, 2t+1) of MMA tile nt are the hi and lo halves of head 4nt + t
+        const int r0 = key_begin + (warp + kScoreWarps * it) * kTileKeys + q, r1 = r0 + 8;
+        const bool v0 = r0 < key_end, v1 = r1 < key_end;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int g = 4 * nt + t;
+            const float y0 = acc[nt][0] + acc[nt][1], y1 = acc[nt][2] + acc[nt][3];
+            if (g < G) {
+                if (v0) { rawu[(int64_t)r0 * G + g] = y0; s1[nt] += y0; s2[nt] = fmaf(y0, y0, s2[nt]); }
+                if (v1) { rawu[(int64_t)r1 * G + g] = y1; s1[nt] += y1; s2[nt] = fmaf(y1, y1, s2[nt]); }
+            }
+        }
+    }
+    if (timed_out) {
+        // a copy did not land within the bound: report it, give copies still in flight one more bounded
+        // chance to land in this block's shared memory, and fall through to the block's normal exit
+        if (p.device_status) atomicExch(p.device_status, TRI_STATUS_TIMEOUT);
+        for (int st = 0; st < kStages; ++st) (void)mbar_wait_bounded(my_bars + st * 8, 0);
+    }
+
+    // ---- per-block (sum, sum^2) in a fixed order: lanes with equal t, then warps ----
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        double a = s1[nt], b = s2[nt];
+#pragma unroll
+        for (int m = 4; m < 32; m <<= 1) {
+            a += __shfl_xor_sync(0xffffffffu, a, m);
+            b += __shfl_xor_sync(0xffffffffu, b, m);
+        }
+        if (q == 0) { red[warp][4 * nt + t][0] = a; red[warp][4 * nt + t][1] = b; }
+    }
+    __syncthreads();
+    if (tid < G) {
+        double a = 0.0, b = 0.0;
+        for (int w = 0; w < kScoreWarps; ++w) { a += red[w][tid][0]; b += red[w][tid][1]; }
+        p.partials[((int64_t)u * p.nchunks + chunk) * G + tid] = make_double2(a, b);
+    }
+}
+
+}  // namespace tri
