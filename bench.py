@@ -35,6 +35,25 @@ DEFAULT_WORKLOAD = "qwen3_8b_oneshot_32k"
 NOMINAL_HBM_GBS = 8000.0
 
 
+# DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum on
+# 1,048,576 keys: 268.564736 MB + 13.445376 MB), valid only for the kernel source it was taken on.
+SCORE_TRAFFIC = {"bytes_per_key": (268564736 + 13445376) / 1048576,
+                 "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
+                             "paper_2604_04921_b200/csrc/tri_common.cuh"],
+                 "sha256": "1fae8a5229be2e5184832882617f8c1545fe0a1908945553fad8315c9ca44fb0"}
+
+
+def score_traffic_per_launch(keys):
+    """ncu traffic scaled to a launch of `keys` keys (it grows in proportion), or None if the kernel's
+    source has changed since the counters were taken."""
+    import hashlib
+    h = hashlib.sha256()
+    for rel in SCORE_TRAFFIC["sources"]:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return SCORE_TRAFFIC["bytes_per_key"] * keys if h.hexdigest() == SCORE_TRAFFIC["sha256"] else None
+
+
 def measured_peaks():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -134,12 +153,29 @@ def sample_units(spec, count):
     return out[:count]
 
 
+def max_over_ranks(ms, dist, device):
+    """The slowest rank's time: MAX all-reduce over the process group (identity without one)."""
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, keys_per_rank_step, ms_step):
+    """Replicas: every rank processes the same number of keys per step; the job's rate is their sum
+    over the slowest rank's step time."""
+    return world * keys_per_rank_step / (ms_step * 1e-3)
+
+
 def run_reference(args, spec):
     """--impl reference: the oracle as it stands, one sampled unit per step, on the host cores."""
     import oracle
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    if args.steps <= 0:
+        args.steps = 4
     oracle.build()
     units = sample_units(spec, args.warmup + args.steps)
     oracle_sample(spec, units[:max(1, min(args.warmup, 1))], spec.budget)     # warm-up: page in, build
@@ -161,7 +197,7 @@ def run_reference(args, spec):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps; 0 = as many as fill about one second")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
@@ -227,6 +263,16 @@ def main():
     for _ in range(args.warmup):
         step()
     barrier()
+    if args.steps <= 0:
+        # fill about one second, so that the clock sampler sees the region under load
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            step()
+        e1.record()
+        barrier()
+        est = max_over_ranks(e0.elapsed_time(e1) / 3, dist, dev)
+        args.steps = int(min(3000, max(20, 1000.0 / est)))
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -236,20 +282,16 @@ def main():
         step()
     e1.record()
     barrier()
-    ms = e0.elapsed_time(e1)
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    ms_step = ms_total / args.steps
+    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
 
     # per-kernel durations: second pass, events recorded by the library between its launches
     ctx.profile_begin()
     per = {k: 0.0 for k in ctx.KERNELS}
-    for _ in range(args.steps):
+    prof_steps = min(args.steps, 200)
+    for _ in range(prof_steps):
         step()
         for k, v in ctx.profile_read().items():
-            per[k] += v / args.steps
+            per[k] += v / prof_steps
     ctx.profile_end()
     clocks = sampler.stop() if rank == 0 else None
 
@@ -257,7 +299,7 @@ def main():
     score_bytes = 256 * keys_per_step
     score_gbs = score_bytes / (per["score"] * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": world * keys_per_step / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_value(world, keys_per_step, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": spec.name + (f"[first {L} layers]" if L != spec.n_layers else ""),
@@ -270,7 +312,7 @@ def main():
                 "frac_of_measured_copy_peak": abytes / (ms_step * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8tbs": abytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
         "roofline": {"kernel": "k_score_tma", "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": score_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(keys_per_step), "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"]},
         "kernel_ms": per,
         "gpu_launches": launches_per_step * args.steps,
@@ -305,14 +347,11 @@ def main():
             step_host()
         e1.record()
         barrier()
-        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if dist is not None:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item()) / e2e_steps
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), dist, dev) / e2e_steps
         assert int(hcnt.min()) == min(B, min(lens))
         h2d = (hk.numel() + hv.numel()) * 2 + (0 if hpos is None else hpos.numel() * 4) + S * 12
         d2h = (hk2.numel() + hv2.numel()) * 2 + hp2.numel() * 4 + U * 4
-        line["e2e"] = {"value": world * keys_per_step / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+        line["e2e"] = {"value": whole_job_value(world, keys_per_step, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                        "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                        "call": "tri_compress_host (pinned host K/V/positions in, compacted K/V/positions/counts out)"}
         del hk, hv, hk2, hv2

@@ -53,12 +53,12 @@ def check_scores(raw_gpu: np.ndarray, s_gpu: np.ndarray, ref: dict):
     sig = raw_o.std(axis=1)
     tol = REL * np.maximum(np.abs(raw_o), sig[:, None])
     err = np.abs(raw_gpu.T.astype(np.float64) - raw_o)
-    assert np.all(err <= tol), f"raw score error {np.max(err / tol):.3g} x tolerance"
+    assert np.all(err <= tol), f"raw score error {np.max(err / np.maximum(tol, 1e-300)):.3g} x tolerance"
     s_o = ref["s_final"]
     tol_s = REL * np.maximum(np.abs(s_o), 1.0)
     err_s = np.abs(s_gpu.astype(np.float64) - s_o)
     assert np.all(err_s <= tol_s), f"final score error {np.max(err_s / tol_s):.3g} x tolerance"
-    return float(np.max(err / tol)), float(np.max(err_s / tol_s))
+    return float(np.max(err / np.maximum(tol, 1e-300))), float(np.max(err_s / tol_s))
 
 
 def check_kept(idx_gpu: np.ndarray, cnt_gpu: int, ref: dict, budget: int):
