@@ -163,6 +163,36 @@ tri_status tri_compress_host(tri_ctx *ctx, const tri_cache_view *src_host, const
                              int32_t *kept_cnt_host, int32_t *kept_cnt_dev,
                              void *ws, size_t ws_bytes, void *stream);
 
+/*
+ * tri_score without a workspace argument (the paper has no counterpart; this is a packaging variant
+ * of tri_score for callers that have nowhere to get scratch memory from at call time).  Examples: an
+ * inference server that gave every spare byte of HBM to its KV page pool at start-up, so that a later
+ * cudaMalloc fails; a plug-in that is handed raw device pointers by a host application and must keep
+ * out of that application's allocator; a latency-critical loop that cannot afford the device-wide
+ * synchronisation an allocation may imply.
+ *
+ * Same arguments, outputs and arithmetic as tri_score, minus ws / ws_bytes.  The phasors, raw scores
+ * and partial sums live in one array of TRI_SCORE_STATIC_SCRATCH_BYTES bytes that is compiled into
+ * the library as a device global: every GPU on which the library's module gets loaded holds those
+ * bytes until the process exits, whether or not this function is ever called.
+ *   - The call needs S*1024 bytes of phasors, U*n_max*G*4 bytes of raw scores and 16*G bytes of
+ *     partial sums per scoring block (about one block per 1,536 keys), U = n_layers*S*n_kv_heads.
+ *     If that exceeds the array the call launches nothing, returns TRI_ERR_WORKSPACE and leaves
+ *     both sizes in tri_last_cuda_error().  With G = 4 the array covers about 1.0 M keys per call
+ *     (e.g. one layer of 8 KV heads at 128 K keys each).
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, which
+ *     may load the module); make that first call during set-up, outside any stream capture.  No call
+ *     allocates or frees device memory, and the context must have been created on the current device.
+ *   - All calls on a device share the one array and it keeps what the last call left.  Nothing in it
+ *     has to start at zero (every word that is read was written earlier in the same call), so it is
+ *     never cleared; but two calls whose kernels overlap on the GPU (different streams, or
+ *     different host threads on different streams) race on it.  Keep them on one stream or order them
+ *     with events.
+ */
+#define TRI_SCORE_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+tri_status tri_score_static(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                            float *scores, float *raw, void *stream);
+
 /* Number of kernel launches one tri_compress call issues for this shape (for launch accounting). */
 int32_t tri_compress_launches(const tri_ctx *ctx, const tri_cache_view *src, const tri_cache_view *dst);
 

@@ -24,7 +24,7 @@ HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cu
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",
-           "tri_compress", "tri_compress_host", "tri_compress_launches", "tri_last_cuda_error",
+           "tri_compress", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_last_cuda_error",
            "tri_profile_begin", "tri_profile_read", "tri_profile_end"]
 
 STATUS = {0: "TRI_OK", 1: "TRI_ERR_INVALID_ARG", 2: "TRI_ERR_UNSUPPORTED", 3: "TRI_ERR_WORKSPACE",
@@ -93,6 +93,8 @@ def lib():
     L.tri_workspace_bytes.restype = sz
     L.tri_score.argtypes = [P, VP, i32, P, P, P, P, sz, P]
     L.tri_score.restype = ctypes.c_int
+    L.tri_score_static.argtypes = [P, VP, i32, P, P, P, P]
+    L.tri_score_static.restype = ctypes.c_int
     L.tri_select.argtypes = [P, P, P, i32, i32, i32, P, P, P, sz, P]
     L.tri_select.restype = ctypes.c_int
     L.tri_compact.argtypes = [P, VP, P, P, i32, i32, VP, P, P]
@@ -227,6 +229,28 @@ class TriContext:
             assert raw.numel() == self.units(S) * cv.n_max * self.group_size
         _check(lib().tri_score(self._h, ctypes.byref(cv), S, _ptr(cur_pos), _ptr(scores), _ptr(raw), _ptr(ws),
                                ws.numel(), _stream()), "tri_score")
+
+    STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+    def score_static(self, src: CacheView, cur_pos: torch.Tensor, scores: torch.Tensor,
+                     raw: Optional[torch.Tensor] = None):
+        """tri_score_static: like score() but with no workspace tensor -- the library's built-in
+        16 MiB device array is the scratch.  For callers that cannot obtain device memory at call
+        time (an engine whose page pool owns all of HBM, a plug-in barred from the host's allocator).
+        This method creates no torch tensor.  Shapes that need more scratch raise TriError(3) with
+        both sizes in the message.  Calls share that array: do not let two of them overlap on the GPU.
+        Make the first call on a device during set-up (it looks up the array's address)."""
+        S = cur_pos.shape[0]
+        cv = src.c_view()
+        assert cur_pos.dtype == torch.int64 and scores.dtype == torch.float32 and scores.is_contiguous()
+        assert scores.numel() == self.units(S) * cv.n_max
+        if raw is not None:
+            assert raw.dtype == torch.float32 and raw.is_contiguous()
+            assert raw.numel() == self.units(S) * cv.n_max * self.group_size
+        code = lib().tri_score_static(self._h, ctypes.byref(cv), S, _ptr(cur_pos), _ptr(scores), _ptr(raw), _stream())
+        if code == 3:
+            raise TriError(code, "tri_score_static", lib().tri_last_cuda_error().decode())
+        _check(code, "tri_score_static")
 
     def select(self, scores: torch.Tensor, seq_lens: torch.Tensor, n_max: int, budget: int,
                kept_idx: torch.Tensor, kept_cnt: torch.Tensor, ws: Optional[torch.Tensor] = None):

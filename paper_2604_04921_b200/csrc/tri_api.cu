@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -528,4 +529,52 @@ extern "C" tri_status tri_profile_end(tri_ctx *c)
     if (c->profiling) for (int i = 0; i < kProfEvents; ++i) cudaEventDestroy(c->ev[i]);
     c->profiling = false;
     return TRI_OK;
+}
+
+// ----------------------------------------------------------------------------------------------
+// tri_score_static: scoring with the workspace in a device global instead of a caller's buffer
+// ----------------------------------------------------------------------------------------------
+// One copy per device that loads this module, held until the process exits.  In host code the name
+// below is only a handle for cudaGetSymbolAddress: it is not a device address and must never be
+// passed to a kernel as one.
+static __device__ __align__(256) unsigned char g_score_scratch[TRI_SCORE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static void *g_score_scratch_addr[kMaxDevices];   // device address of g_score_scratch, per device, once looked up
+static std::mutex g_score_scratch_mu;
+
+// Device address of the scratch array on the current device; the first call per device asks the runtime.
+static tri_status score_scratch_address(int dev, void **out)
+{
+    std::lock_guard<std::mutex> lock(g_score_scratch_mu);
+    if (!g_score_scratch_addr[dev]) {
+        void *p = nullptr;
+        TRI_CUDA(cudaGetSymbolAddress(&p, g_score_scratch));
+        if (!p) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_score_scratch)");
+        g_score_scratch_addr[dev] = p;
+    }
+    *out = g_score_scratch_addr[dev];
+    return TRI_OK;
+}
+
+extern "C" tri_status tri_score_static(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                       float *scores, float *raw, void *stream)
+{
+    tri_status r;
+    if (!c || !src || !cur_pos || !scores) return TRI_ERR_INVALID_ARG;
+    if ((r = check_view(src, true)) != TRI_OK) return r;
+    if ((r = check_common(c, S, src->n_max, 1)) != TRI_OK) return r;
+    Plan pl = make_plan(c, S, src->n_max, 0);
+    const size_t need = pl.off_scores;           // phasors + raw scores + partial sums; scores go to the caller
+    if (need > (size_t)TRI_SCORE_STATIC_SCRATCH_BYTES) {
+        snprintf(g_err, sizeof g_err, "tri_score_static: this shape needs %zu bytes of scratch, the built-in array holds %zu",
+                 need, (size_t)TRI_SCORE_STATIC_SCRATCH_BYTES);
+        return TRI_ERR_WORKSPACE;
+    }
+    int dev = -1;
+    TRI_CUDA(cudaGetDevice(&dev));
+    if (dev != c->device || dev < 0 || dev >= kMaxDevices) return TRI_ERR_INVALID_ARG;
+    void *ws = nullptr;
+    if ((r = score_scratch_address(dev, &ws)) != TRI_OK) return r;
+    return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream);
 }
