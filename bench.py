@@ -69,17 +69,26 @@ class ClockSampler:
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.proc, self.first = index, [], None, 0
 
     def start(self):
+        """Starts nvidia-smi and waits for its first sample: its start-up can stall the GPU for seconds and
+        must not fall into a timed region."""
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
+            t0 = time.time()
+            while not self.rows and time.time() - t0 < 30.0 and self.proc.poll() is None:
+                time.sleep(0.05)
         except Exception:
             self.proc = None
+
+    def mark(self):
+        """Samples taken from now on count (call right before the timed region)."""
+        self.first = len(self.rows)
 
     def _read(self):
         for line in self.proc.stdout:
@@ -88,7 +97,7 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.06)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -96,7 +105,7 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for r in self.rows[self.first:]:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
             except Exception:
@@ -260,6 +269,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(args.warmup):
         step()
     barrier()
@@ -273,15 +285,14 @@ def main():
         barrier()
         est = max_over_ranks(e0.elapsed_time(e1) / 3, dist, dev)
         args.steps = int(min(3000, max(20, 1000.0 / est)))
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    sampler.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
+    clocks = sampler.stop() if rank == 0 else None
     ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
 
     # per-kernel durations: second pass, events recorded by the library between its launches
@@ -293,7 +304,6 @@ def main():
         for k, v in ctx.profile_read().items():
             per[k] += v / prof_steps
     ctx.profile_end()
-    clocks = sampler.stop() if rank == 0 else None
 
     peak, peak_src = measured_peaks()
     score_bytes = 256 * keys_per_step

@@ -354,11 +354,18 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
     p.k_vec = kHeadDim * p.k_esize / 16;
     p.v_vec = (src->v && dst->v) ? kHeadDim * 2 / 16 : 0;
     p.device_status = device_status;
+    const bool rows16 = src->k_kind == 0 && p.v_vec != 0;     // bf16 K and V: the row-gather kernel applies
+    dim3 grid(U, (budget + kFastRowsPerBlock - 1) / kFastRowsPerBlock);
     if (aliases(src, dst)) {
-        k_compact_inplace<<<U, kInplaceThreads, 0, st>>>(p);
+        // in place: the prefix whose sources lie inside the destination range goes tile by tile in one block
+        // per unit; everything behind it is a hazard-free gather
+        k_compact_inplace<<<U, kInplaceThreads, 0, st>>>(p, rows16 ? 1 : 0);
+        if (rows16) k_gather_rows<true><<<grid, kGatherThreads, 0, st>>>(p);
+    } else if (rows16) {
+        k_gather_rows<false><<<grid, kGatherThreads, 0, st>>>(p);
     } else {
-        dim3 grid(U, (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock);
-        k_gather<<<grid, kGatherThreads, 0, st>>>(p);
+        dim3 grid_any(U, (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock);
+        k_gather_any<<<grid_any, kGatherThreads, 0, st>>>(p);
     }
     tri_status r = check_launch("k_compact");
     mark(c, 5, st);
@@ -452,8 +459,11 @@ extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_
 
 extern "C" int32_t tri_compress_launches(const tri_ctx *c, const tri_cache_view *src, const tri_cache_view *dst)
 {
-    (void)c; (void)src; (void)dst;
-    return 5;   // fold, score, normalise, select, gather
+    (void)c;
+    if (!src || !dst) return 0;
+    // fold, score, normalise, select, gather; an in-place round of bf16 K + V splits the gather into the tiled
+    // prefix pass and the parallel pass behind it
+    return 5 + ((aliases(src, dst) && src->k_kind == 0 && src->v && dst->v) ? 1 : 0);
 }
 
 extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_host, const tri_cache_view *src_dev,

@@ -37,9 +37,78 @@ __device__ __forceinline__ void st_once(void *p, uint4 v)
                  : "memory");
 }
 
-// Out-of-place gather.  grid = (U, ceil(budget / 64)); a warp moves 8 rows at a time, lanes 0..15
-// carry the K row and lanes 16..31 the V row (bf16), so every access is a full 256-byte row.
-__global__ void __launch_bounds__(kGatherThreads) k_gather(const CompactParams p)
+// Gather of bf16 K and V rows (the common case), contiguous or paged on either side.
+// grid = (U, ceil(budget / kFastRowsPerBlock)).  Lanes 0..15 of a warp carry a K row and lanes 16..31
+// the V row of the same slot, 16 bytes each, so every access is a whole 256-byte row.  A warp keeps
+// kFastRows rows in flight (all loads issued before the first store) and walks kFastIters such groups.
+// Lane r < kFastRows resolves the addresses of row r of the group (index load, page-table lookups) and
+// hands them to the other lanes by shuffle, so the address work is done once per row, not per lane;
+// that keeps the kernel at 64 registers, four blocks per SM.
+//
+// AFTER_PREFIX = true is the second phase of an in-place compaction: it moves only the row tiles that
+// k_compact_inplace left alone (tiles whose first source lies at or beyond the kept count), whose sources
+// are all outside the destination range [0, count) -- see k_compact_inplace.
+constexpr int kFastRows = 8;
+constexpr int kFastIters = 2;
+constexpr int kFastRowsPerBlock = kGatherWarps * kFastRows * kFastIters;
+constexpr int kInplaceRows = 32;        // rows per tile of the in-place schedule
+
+template <bool AFTER_PREFIX>
+__global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const CompactParams p)
+{
+    const int u = blockIdx.x;
+    const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
+    const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
+    if (!AFTER_PREFIX && blockIdx.y == 0 && threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0)
+        p.new_seq_lens[s] = cnt;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int jw = blockIdx.y * kFastRowsPerBlock + warp * (kFastRows * kFastIters);
+    if (jw >= cnt) return;
+    const int32_t *idx = p.kept_idx + (int64_t)u * p.budget;
+    const bool is_v = lane >= 16;
+    const char *sb = (is_v ? p.src.v : p.src.k) + (lane & 15) * 16;
+    char *db = (is_v ? p.dst.v : p.dst.k) + (lane & 15) * 16;
+    const int n_src = p.src.n_max;
+
+#pragma unroll 1
+    for (int it = 0; it < kFastIters; ++it) {
+        const int j0 = jw + it * kFastRows;
+        if (j0 >= cnt) break;
+        if (AFTER_PREFIX && __ldg(idx + (j0 & ~(kInplaceRows - 1))) < cnt) continue;   // the first phase moved this tile
+        // lane r resolves row j0 + r; rows past the count, indices outside the unit and bad page ids are skipped
+        int mine = -1;
+        int64_t so = -1, dof = -1;
+        if (lane < kFastRows && j0 + lane < cnt) {
+            mine = __ldg(idx + j0 + lane);
+            if (mine >= 0 && mine < n_src) {
+                so = row_offset(p.src, l, s, h, mine);
+                dof = row_offset(p.dst, l, s, h, j0 + lane);
+            }
+            if (so < 0 || dof < 0) {
+                if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
+                mine = -1; so = -1; dof = -1;
+            }
+        }
+        uint4 val[kFastRows];
+#pragma unroll
+        for (int r = 0; r < kFastRows; ++r) {
+            const int64_t o = __shfl_sync(0xffffffffu, so, r);
+            if (o >= 0) val[r] = ld_once(sb + o * 2);
+        }
+#pragma unroll
+        for (int r = 0; r < kFastRows; ++r) {
+            const int64_t o = __shfl_sync(0xffffffffu, dof, r);
+            if (o >= 0) st_once(db + o * 2, val[r]);
+        }
+        if (p.dst.positions && mine >= 0)
+            p.dst.positions[(int64_t)u * p.dst.n_max + j0 + lane] =
+                p.src.positions ? p.src.positions[(int64_t)u * p.src.n_max + mine] : mine;
+    }
+}
+
+// Out-of-place gather for the remaining cases (fp32 keys, no value cache).
+// grid = (U, ceil(budget / 64)); a warp moves 8 rows at a time, 16 bytes per lane.
+__global__ void __launch_bounds__(kGatherThreads) k_gather_any(const CompactParams p)
 {
     const int u = blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
@@ -101,11 +170,16 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather(const CompactParams p
 // In-place (or aliasing) compaction: one block per unit walks the kept rows in ascending tiles.
 // Every row of a tile is staged in shared memory before any row of the tile is written; since
 // kept_idx[j] >= j and is increasing, a tile's destinations lie strictly below every source of the
-// following tiles, so no source is overwritten before it has been read.
+// following tiles, so no source is overwritten before it has been read.  Rows already in their slot
+// (kept_idx[j] == j) are not touched.
+//
+// prefix_only = 1 stops at the first tile whose first source index is >= the kept count: from there on
+// every source lies outside the destination range [0, count), nothing can be overwritten before it is
+// read, and k_gather_rows<true> moves those tiles with full parallelism in a following launch (its
+// destinations, >= the prefix end, are never sources of the prefix, whose sources were all read here first).
 constexpr int kInplaceThreads = 512;
-constexpr int kInplaceRows = 32;        // rows per tile: 32 x (512 B K + 256 B V) <= 24 KB
 
-__global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace(const CompactParams p)
+__global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace(const CompactParams p, const int prefix_only)
 {
     __shared__ uint4 stage[kInplaceRows * 48];
     __shared__ int32_t pos_s[kInplaceRows];
@@ -117,10 +191,12 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace(const Compa
     const int per_row = p.k_vec + p.v_vec;
 
     for (int j0 = 0; j0 < cnt; j0 += kInplaceRows) {
+        if (prefix_only && __ldg(idx + j0) >= cnt) break;
         const int rows = min(kInplaceRows, cnt - j0);
         for (int i = threadIdx.x; i < rows * per_row; i += kInplaceThreads) {
             int r = i / per_row, c = i - r * per_row;
             int srow = __ldg(idx + j0 + r);
+            if (srow == j0 + r) continue;                      // already in its slot
             int64_t so = (srow >= 0 && srow < p.src.n_max) ? row_offset(p.src, l, s, h, srow) : -1;
             const bool is_k = c < p.k_vec;
             uint4 v = make_uint4(0, 0, 0, 0);
@@ -136,6 +212,7 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace(const Compa
         __syncthreads();
         for (int i = threadIdx.x; i < rows * per_row; i += kInplaceThreads) {
             int r = i / per_row, c = i - r * per_row;
+            if (__ldg(idx + j0 + r) == j0 + r) continue;
             int64_t dof = row_offset(p.dst, l, s, h, j0 + r);
             const bool is_k = c < p.k_vec;
             if (dof < 0) { if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK); }

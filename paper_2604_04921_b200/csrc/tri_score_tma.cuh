@@ -21,9 +21,9 @@
 
 namespace tri {
 
-constexpr int kStages = 3;
+constexpr int kStages = 2;
 constexpr int kTileBytes = kTileKeys * kHeadDim * 2;                       // 4096
-constexpr int kScoreDynSmem = kScoreWarps * kStages * kTileBytes;          // 98304
+constexpr int kScoreDynSmem = kScoreWarps * kStages * kTileBytes;          // 65536: three blocks per SM
 constexpr uint32_t kWaitPolls = 1u << 22;                                  // bound on every mbarrier wait
 constexpr int TRI_STATUS_TIMEOUT = 6;
 
@@ -92,7 +92,7 @@ __device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x 
 __device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 
 template <int NT, int LAYOUT>
-__global__ void __launch_bounds__(kScoreThreads)
+__global__ void __launch_bounds__(kScoreThreads, 3)
 k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
 {
     extern __shared__ __align__(1024) uint8_t tiles[];   // [warp][stage][half][16 rows][128 B]
