@@ -275,7 +275,8 @@ tri_status launch_score_tma(int NT, dim3 grid, cudaStream_t st, const CUtensorMa
     return launch_score_tma_one<4, LAYOUT>(grid, st, map, sp);
 }
 
-// fold -> raw scores -> z-score/max.  3 launches.
+// fold -> raw scores -> z-score/max (3 launches); without the last one when `scores` is NULL: the fused round
+// leaves the normalisation to its selection kernel.
 tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, float *scores,
                      float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st)
 {
@@ -312,6 +313,10 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     }
     if ((r = check_launch("k_score")) != TRI_OK) return r;
     mark(c, 2, st);
+    if (!scores) {
+        mark(c, 3, st);
+        return TRI_OK;
+    }
 
     NormParams np;
     np.raw = raw; np.partials = part; np.seq_lens = src->seq_lens; np.scores = scores;
@@ -323,15 +328,29 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     return r;
 }
 
+// Top-B selection.  pl == NULL: from the final scores in `scores` (tri_select).  pl != NULL: the fused round,
+// straight from the raw scores and partial sums in the workspace `ws`; final scores are parked in its score area.
 tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
                       int32_t budget, int32_t *kept_idx, int32_t *kept_cnt, int32_t *new_seq_lens,
-                      int32_t U, cudaStream_t st)
+                      int32_t U, const Plan *pl, char *ws, cudaStream_t st)
 {
     SelectParams p;
-    p.scores = scores; p.seq_lens = seq_lens; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
+    p.scores = scores; p.scores_w = nullptr; p.seq_lens = seq_lens; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
     p.new_seq_lens = new_seq_lens;
     p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget;
-    k_select<<<U, kSelThreads, 0, st>>>(p);
+    p.raw = nullptr; p.partials = nullptr; p.G = c->desc.group_size; p.chunk = 0; p.nchunks = 0;
+    if (pl) {
+        p.scores_w = (float *)(ws + pl->off_scores);
+        p.scores = p.scores_w;
+        p.raw = (const float *)(ws + pl->off_raw);
+        p.partials = (const double2 *)(ws + pl->off_part);
+        p.chunk = pl->chunk; p.nchunks = pl->nchunks;
+        if (n_max <= kSelSmallUnit) k_select<true, 256><<<U, 256, 0, st>>>(p);
+        else k_select<true, 1024><<<U, 1024, 0, st>>>(p);
+    } else {
+        if (n_max <= kSelSmallUnit) k_select<false, 256><<<U, 256, 0, st>>>(p);
+        else k_select<false, 1024><<<U, 1024, 0, st>>>(p);
+    }
     tri_status r = check_launch("k_select");
     mark(c, 4, st);
     return r;
@@ -408,12 +427,13 @@ extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t 
                                  int32_t n_max, int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
                                  void *ws, size_t ws_bytes, void *stream)
 {
-    (void)ws; (void)ws_bytes;   // the selection keeps its histograms in shared memory
+    (void)ws; (void)ws_bytes;   // the selection keeps its histograms and candidates in shared memory
     tri_status r;
     if (!c || !scores || !seq_lens || !kept_idx || !kept_cnt) return TRI_ERR_INVALID_ARG;
     if ((r = check_common(c, S, n_max, budget)) != TRI_OK) return r;
     int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
-    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, nullptr, U, (cudaStream_t)stream);
+    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, nullptr, U, nullptr, nullptr,
+                      (cudaStream_t)stream);
 }
 
 extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx,
@@ -448,11 +468,11 @@ extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_
     if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char *w = (char *)ws;
-    float *scores = (float *)(w + pl.off_scores);
     int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
     int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
-    if ((r = run_score(c, src, S, cur_pos, scores, nullptr, w, pl, device_status, st)) != TRI_OK) return r;
-    if ((r = run_select(c, scores, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, st)) != TRI_OK)
+    if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st)) != TRI_OK) return r;
+    if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, &pl, w, st)) !=
+        TRI_OK)
         return r;
     return run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, pl.U, st);
 }
@@ -461,9 +481,9 @@ extern "C" int32_t tri_compress_launches(const tri_ctx *c, const tri_cache_view 
 {
     (void)c;
     if (!src || !dst) return 0;
-    // fold, score, normalise, select, gather; an in-place round of bf16 K + V splits the gather into the tiled
-    // prefix pass and the parallel pass behind it
-    return 5 + ((aliases(src, dst) && src->k_kind == 0 && src->v && dst->v) ? 1 : 0);
+    // fold, score, select (which also normalises), gather; an in-place round of bf16 K + V splits the gather into
+    // the tiled prefix pass and the parallel pass behind it
+    return 4 + ((aliases(src, dst) && src->k_kind == 0 && src->v && dst->v) ? 1 : 0);
 }
 
 extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_host, const tri_cache_view *src_dev,

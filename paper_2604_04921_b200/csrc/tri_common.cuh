@@ -41,10 +41,11 @@ __device__ __forceinline__ int64_t row_offset(const View &w, int l, int s, int h
            (int64_t)(n - pg * w.page_size) * w.stride_slot;
 }
 
-// Order-preserving image of an fp32 in uint32: a > b  <=>  key(a) > key(b) (for non-NaN values).
+// Order-preserving image of an fp32 in uint32: a > b  <=>  key(a) > key(b) (for non-NaN values); -0.0 and
+// +0.0 are equal scores and get the same image.  Never 0 for a non-NaN input.
 __device__ __forceinline__ uint32_t float_key(float x)
 {
-    uint32_t b = __float_as_uint(x);
+    uint32_t b = __float_as_uint(x + 0.0f);          // -0.0 + 0.0 = +0.0
     return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
 }
 

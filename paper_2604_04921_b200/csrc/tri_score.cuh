@@ -188,6 +188,50 @@ k_score_f32_pre(const ScoreParams p, const double *__restrict__ omega, const dou
     }
 }
 
+// mu_g and 1/sigma_g of one unit from the per-block partial sums, added in a fixed order so that every
+// block (and every kernel) that asks gets the same bits.  Threads 0 .. 255 of the block take part:
+// 16 lanes per head, lane i adds blocks i, i+16, ...; then a fixed butterfly.  Results land in shared
+// memory; the caller synchronises.  A head whose scores are equal up to fp32 resolution gets 1/sigma = 0
+// (it then contributes z = 0: Section 4.3 with sigma_g = 0).
+__device__ __forceinline__ void unit_mean_rstd(const double2 *__restrict__ part, int G, int used, int n,
+                                               float *mu_s, float *rs_s)
+{
+    const int tid = threadIdx.x;
+    if (tid >= 16 * kMaxGroup) return;          // whole warps only: the shuffles below stay converged
+    int g = tid >> 4, i = tid & 15;
+    double a = 0.0, b = 0.0;
+    if (g < G)
+        for (int c = i; c < used; c += 16) {
+            double2 v = part[(int64_t)c * G + g];
+            a += v.x;
+            b += v.y;
+        }
+    for (int m = 1; m < 16; m <<= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, m);
+        b += __shfl_xor_sync(0xffffffffu, b, m);
+    }
+    if (g < G && i == 0) {
+        double mu = a / (double)n;
+        double var = b / (double)n - mu * mu;
+        double rs = (var > 1e-12 * mu * mu && var > 0.0) ? rsqrt(var) : 0.0;
+        mu_s[g] = (float)mu;
+        rs_s[g] = (float)rs;
+    }
+}
+
+// z-score + max over the group for one key (Section 4.3), from its G raw scores.
+__device__ __forceinline__ float zmax4(float4 x, const float *mu_s, const float *rs_s)
+{
+    return fmaxf(fmaxf((x.x - mu_s[0]) * rs_s[0], (x.y - mu_s[1]) * rs_s[1]),
+                 fmaxf((x.z - mu_s[2]) * rs_s[2], (x.w - mu_s[3]) * rs_s[3]));
+}
+__device__ __forceinline__ float zmax(const float *row, int G, const float *mu_s, const float *rs_s)
+{
+    float z = -INFINITY;
+    for (int g = 0; g < G; ++g) z = fmaxf(z, (row[g] - mu_s[g]) * rs_s[g]);
+    return z;
+}
+
 // ---------------------------------------------------------------------------------------
 // GQA normalise-then-aggregate (Section 4.3): S_final(k) = max_g (raw_g(k) - mu_g) / sigma_g.
 // Same grid as the scoring kernel.  mu, sigma come from the per-block partial sums, added in a
@@ -213,46 +257,16 @@ __global__ void __launch_bounds__(256) k_normalize(const NormParams p)
     const int key_end = min(key_begin + p.chunk, n);
     const int G = p.G;
     const int used = (n + p.chunk - 1) / p.chunk;
-    {
-        // 16 lanes per head: lane i adds blocks i, i+16, ...; then a fixed butterfly
-        int g = tid >> 4, i = tid & 15;
-        double a = 0.0, b = 0.0;
-        if (g < G)
-            for (int c = i; c < used; c += 16) {
-                double2 v = p.partials[((int64_t)u * p.nchunks + c) * G + g];
-                a += v.x;
-                b += v.y;
-            }
-        for (int m = 1; m < 16; m <<= 1) {
-            a += __shfl_xor_sync(0xffffffffu, a, m);
-            b += __shfl_xor_sync(0xffffffffu, b, m);
-        }
-        if (g < G && i == 0) {
-            double mu = a / (double)n;
-            double var = b / (double)n - mu * mu;
-            // scores equal up to fp32 resolution: sigma = 0, the head contributes z = 0
-            double rs = (var > 1e-12 * mu * mu && var > 0.0) ? rsqrt(var) : 0.0;
-            mu_s[g] = (float)mu;
-            rs_s[g] = (float)rs;
-        }
-    }
+    unit_mean_rstd(p.partials + (int64_t)u * p.nchunks * G, G, used, n, mu_s, rs_s);
     __syncthreads();
     const float *rawu = p.raw + (int64_t)u * p.n_max * G;
     float *out = p.scores + (int64_t)u * p.n_max;
     if (G == 4) {
-        const float m0 = mu_s[0], m1 = mu_s[1], m2 = mu_s[2], m3 = mu_s[3];
-        const float r0 = rs_s[0], r1 = rs_s[1], r2 = rs_s[2], r3 = rs_s[3];
-        for (int key = key_begin + tid; key < key_end; key += 256) {
-            float4 x = *reinterpret_cast<const float4 *>(rawu + (int64_t)key * 4);
-            float z = fmaxf(fmaxf((x.x - m0) * r0, (x.y - m1) * r1), fmaxf((x.z - m2) * r2, (x.w - m3) * r3));
-            out[key] = z;
-        }
+        for (int key = key_begin + tid; key < key_end; key += 256)
+            out[key] = zmax4(*reinterpret_cast<const float4 *>(rawu + (int64_t)key * 4), mu_s, rs_s);
     } else {
-        for (int key = key_begin + tid; key < key_end; key += 256) {
-            float z = -INFINITY;
-            for (int g = 0; g < G; ++g) z = fmaxf(z, (rawu[(int64_t)key * G + g] - mu_s[g]) * rs_s[g]);
-            out[key] = z;
-        }
+        for (int key = key_begin + tid; key < key_end; key += 256)
+            out[key] = zmax(rawu + (int64_t)key * G, G, mu_s, rs_s);
     }
 }
 

@@ -1,28 +1,56 @@
-// Top-B retention (Section 4.3): exact radix threshold on the order-preserving uint32 image of the
-// fp32 scores, then an index-ordered emit.  One thread block per unit; everything but the scores
-// themselves lives in shared memory, so the pass needs no global scratch.
+// Top-B retention (Section 4.3), exact, one block per unit: 1,024 threads, or 256 for units of up to 8,192 keys
+// (more blocks per SM hide the latency of the short sweeps better).
+//
+//   1. value histogram: final scores are z-scores, so a monotone map onto 2048 steps of 1/128 over
+//      [-8, 8) spreads a unit's keys over hundreds of bins (the top bits of the fp32 image would send
+//      nearly all of them to a dozen bins and serialise the shared-memory atomics).  A top-down scan
+//      of the histogram gives the bin that holds the budget-th largest score.
+//   2. the keys of that bin -- typically a fraction of a percent -- go to a candidate list in shared
+//      memory; an 11 + 11 + 10 bit radix over the list's order-preserving uint32 images gives the exact
+//      threshold key T and how many keys equal to T are kept.  If the list overflows (a unit full of
+//      equal scores, say) the same radix sweeps the unit's keys instead.
+//   3. emit in index order: the unit is cut into spans of at most 32 keys per thread; inside a span warp w
+//      owns a contiguous run of keys, 32 at a time, so warp ballots are already in index order and one
+//      block-wide scan of the warp totals per span places every kept slot.
+//
+// FUSED = true folds the GQA normalise-then-aggregate step into sweep 1: the final score is computed from
+// the raw per-head scores and the unit's (mu_g, 1/sigma_g), parked in the score buffer for the later
+// sweeps (which hit L2), and the round needs no separate normalisation launch.
 #pragma once
-#include "tri_common.cuh"
+#include "tri_score.cuh"
 
 namespace tri {
 
-constexpr int kSelThreads = 1024;
-constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelBins = 2048;
-constexpr int kEmitPerThread = 4;
+constexpr int kSelCand = 4096;                   // candidate list entries
+constexpr int kSelSmallUnit = 8192;              // units up to this many keys take the 256-thread block
 
 struct SelectParams {
-    const float *scores;      // [U][n_max]
+    const float *scores;      // [U][n_max]   final scores: input (FUSED = false) or parked here by sweep 1
+    float *scores_w;          // the same buffer, writable (FUSED = true)
     const int32_t *seq_lens;  // [S]
     int32_t *kept_idx;        // [U][budget]
     int32_t *kept_cnt;        // [U]
     int32_t *new_seq_lens;    // [S] or NULL
     int32_t S, H, n_max, budget;
+    // FUSED only: raw scores and partial sums of the scoring kernel
+    const float *raw;         // [U][n_max][G]
+    const double2 *partials;  // [U][nchunks][G]
+    int32_t G, chunk, nchunks;
 };
 
-// Exclusive prefix sum of `v` over the block's threads (thread order); *total gets the block sum.
+// Monotone map of a score onto 2048 bins: steps of 1/128 over [-8, 8), everything else in the end bins.
+__device__ __forceinline__ uint32_t value_bin(float x)
+{
+    return (uint32_t)min(max(__float2int_rd(fmaf(x, 128.f, 1024.f)), 0), kSelBins - 1);
+}
+
+// Exclusive prefix sum of `v` over the block's THREADS threads (thread order); *total gets the block sum.
+// warp_sums holds 33 words.
+template <int THREADS>
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *warp_sums, uint32_t *total)
 {
+    constexpr int W = THREADS / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = v;
 #pragma unroll
@@ -33,13 +61,13 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *warp_s
     if (lane == 31) warp_sums[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        uint32_t w = warp_sums[lane], winc = w;
+        uint32_t w = lane < W ? warp_sums[lane] : 0u, winc = w;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             uint32_t y = __shfl_up_sync(0xffffffffu, winc, d);
             if (lane >= d) winc += y;
         }
-        warp_sums[lane] = winc - w;            // exclusive warp offsets
+        if (lane < W) warp_sums[lane] = winc - w;   // exclusive warp offsets
         if (lane == 31) warp_sums[32] = winc;  // block total
     }
     __syncthreads();
@@ -49,13 +77,39 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t *warp_s
     return r;
 }
 
-__global__ void __launch_bounds__(kSelThreads) k_select(const SelectParams p)
+// The bin holding the `need`-th largest entry of hist (counted from the top) -> *sel_bin, and how many
+// entries are still needed from that bin -> *sel_need.  Thread t owns the 2048 / THREADS bins from
+// 2047 - t * (2048 / THREADS) downwards.
+template <int THREADS>
+__device__ __forceinline__ void find_bin(const uint32_t *hist, uint32_t need, uint32_t *warp_sums, uint32_t *sel_bin,
+                                         uint32_t *sel_need)
 {
-    __shared__ uint32_t hist[kSelBins];
-    __shared__ uint32_t warp_sums[33];
-    __shared__ uint32_t sel_bin, sel_need;
+    constexpr int BPT = kSelBins / THREADS;
+    const int top = kSelBins - 1 - BPT * (int)threadIdx.x;
+    uint32_t c[BPT], sum = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) { c[q] = hist[top - q]; sum += c[q]; }
+    uint32_t total;
+    uint32_t above = block_excl_scan<THREADS>(sum, warp_sums, &total);   // entries in strictly higher bins
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) {
+        if (above < need && need <= above + c[q]) { *sel_bin = top - q; *sel_need = need - above; }
+        above += c[q];
+    }
+    __syncthreads();
+}
 
-    const int tid = threadIdx.x;
+template <bool FUSED, int THREADS>
+__global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const SelectParams p)
+{
+    constexpr int kSelThreads = THREADS;
+    __shared__ uint32_t hist[kSelBins];
+    __shared__ uint32_t cand[kSelCand];
+    __shared__ uint32_t warp_sums[33];
+    __shared__ uint32_t sel_bin, sel_need, ncand;
+    __shared__ float mu_s[kMaxGroup], rs_s[kMaxGroup];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int u = blockIdx.x;
     const int s = (u / p.H) % p.S;
     const int n = min(__ldg(p.seq_lens + s), p.n_max);
@@ -71,27 +125,73 @@ __global__ void __launch_bounds__(kSelThreads) k_select(const SelectParams p)
         return;
     }
 
-    // ---- threshold: the budget-th largest key, 11 + 11 + 10 bits at a time ----
-    uint32_t prefix = 0, pmask = 0, need = (uint32_t)p.budget;
+    // ---- sweep 1: value histogram (and, fused, the final scores themselves) ----
+    for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
+    if (tid == 0) ncand = 0;
+    if (FUSED) unit_mean_rstd(p.partials + (int64_t)u * p.nchunks * p.G, p.G, (n + p.chunk - 1) / p.chunk, n, mu_s, rs_s);
+    __syncthreads();
+    if (FUSED) {
+        const float *rawu = p.raw + (int64_t)u * p.n_max * p.G;
+        float *scw = p.scores_w + (int64_t)u * p.n_max;
+        if (p.G == 4) {
+#pragma unroll 8
+            for (int i = tid; i < n; i += kSelThreads) {
+                const float z = zmax4(*reinterpret_cast<const float4 *>(rawu + (int64_t)i * 4), mu_s, rs_s);
+                scw[i] = z;
+                atomicAdd(&hist[value_bin(z)], 1u);
+            }
+        } else {
+            for (int i = tid; i < n; i += kSelThreads) {
+                const float z = zmax(rawu + (int64_t)i * p.G, p.G, mu_s, rs_s);
+                scw[i] = z;
+                atomicAdd(&hist[value_bin(z)], 1u);
+            }
+        }
+    } else {
+#pragma unroll 8
+        for (int i = tid; i < n; i += kSelThreads) atomicAdd(&hist[value_bin(sc[i])], 1u);
+    }
+    __syncthreads();                            // histogram complete; parked scores visible to the whole block
+    find_bin<THREADS>(hist, (uint32_t)p.budget, warp_sums, &sel_bin, &sel_need);
+    const uint32_t vb = sel_bin;
+    uint32_t need = sel_need;                   // keys still to take from value bin vb
+
+    // ---- sweep 2: the keys of bin vb become the candidate list ----
+#pragma unroll 8
+    for (int i = tid; i < n; i += kSelThreads) {
+        const float x = sc[i];
+        if (value_bin(x) == vb) {
+            const uint32_t pos = atomicAdd(&ncand, 1u);
+            if (pos < (uint32_t)kSelCand) cand[pos] = float_key(x);
+        }
+    }
+    __syncthreads();
+    const uint32_t nc = ncand;
+    const bool fits = nc <= (uint32_t)kSelCand;
+
+    // ---- the exact key of rank `need` inside bin vb, 11 + 11 + 10 bits at a time ----
+    uint32_t prefix = 0, pmask = 0;
 #pragma unroll 1
     for (int pass = 0; pass < 3; ++pass) {
         const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
         const uint32_t bmask = pass == 2 ? 1023u : 2047u;
         for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
         __syncthreads();
-        for (int i = tid; i < n; i += kSelThreads) {
-            uint32_t k = float_key(sc[i]);
-            if ((k & pmask) == prefix) atomicAdd(&hist[(k >> shift) & bmask], 1u);
+        if (fits) {
+            for (uint32_t i = tid; i < nc; i += kSelThreads) {
+                const uint32_t k = cand[i];
+                if ((k & pmask) == prefix) atomicAdd(&hist[(k >> shift) & bmask], 1u);
+            }
+        } else {
+#pragma unroll 4
+            for (int i = tid; i < n; i += kSelThreads) {
+                const float x = sc[i];
+                const uint32_t k = float_key(x);
+                if (value_bin(x) == vb && (k & pmask) == prefix) atomicAdd(&hist[(k >> shift) & bmask], 1u);
+            }
         }
         __syncthreads();
-        // thread t owns bins 2t', 2t'+1 counted from the top: t' = 1023 - t
-        const int hi_bin = kSelBins - 1 - 2 * tid, lo_bin = hi_bin - 1;
-        const uint32_t ch = hist[hi_bin], cl = hist[lo_bin];
-        uint32_t total;
-        uint32_t above = block_excl_scan(ch + cl, warp_sums, &total);   // keys in strictly higher bins
-        if (above < need && need <= above + ch) { sel_bin = hi_bin; sel_need = need - above; }
-        else if (above + ch < need && need <= above + ch + cl) { sel_bin = lo_bin; sel_need = need - above - ch; }
-        __syncthreads();
+        find_bin<THREADS>(hist, need, warp_sums, &sel_bin, &sel_need);
         prefix |= sel_bin << shift;
         pmask |= bmask << shift;
         need = sel_need;
@@ -100,34 +200,40 @@ __global__ void __launch_bounds__(kSelThreads) k_select(const SelectParams p)
     const uint32_t T = prefix;     // key of the budget-th largest score; `need` keys equal to T are kept
 
     // ---- emit kept slots in ascending order; among keys equal to T the lowest slots win ----
+    // J keys per thread and span (at most 32, fewer for short units so that no sweep runs empty)
+    const uint32_t lt = (1u << lane) - 1u;
+    const int J = min(32, (n + kSelThreads - 1) / kSelThreads);
     uint32_t base = 0, need_rem = need;
-    for (int start = 0; start < n; start += kSelThreads * kEmitPerThread) {
-        const int i0 = start + tid * kEmitPerThread;
-        uint32_t gt = 0, eq = 0, fl_gt = 0, fl_eq = 0;
-#pragma unroll
-        for (int j = 0; j < kEmitPerThread; ++j) {
-            int i = i0 + j;
-            if (i < n) {
-                uint32_t k = float_key(sc[i]);
-                if (k > T) { fl_gt |= 1u << j; ++gt; }
-                else if (k == T) { fl_eq |= 1u << j; ++eq; }
-            }
+#pragma unroll 1
+    for (int span = 0; span < n; span += kSelThreads * J) {
+        const int ibase = span + warp * (32 * J) + lane;
+        uint32_t m_gt = 0, m_eq = 0, w_gt = 0, w_eq = 0;     // bit j: key ibase + 32 j is above / equal to T
+#pragma unroll 4
+        for (int j = 0; j < J; ++j) {
+            const int i = ibase + 32 * j;
+            const uint32_t k = i < n ? float_key(sc[i]) : 0u;  // 0 is below every real key
+            const bool g = k > T, e = k == T;
+            m_gt |= (uint32_t)g << j;
+            m_eq |= (uint32_t)e << j;
+            w_gt += __popc(__ballot_sync(0xffffffffu, g));
+            w_eq += __popc(__ballot_sync(0xffffffffu, e));
         }
+        // a span holds at most 32,768 keys, so the two 16-bit halves never carry into each other
         uint32_t total;
-        uint32_t pre = block_excl_scan(gt | (eq << 16), warp_sums, &total);
+        uint32_t pre = block_excl_scan<THREADS>(lane == 0 ? (w_gt | (w_eq << 16)) : 0u, warp_sums, &total);
+        pre = __shfl_sync(0xffffffffu, pre, 0);
         uint32_t gt_before = pre & 0xffffu, eq_before = pre >> 16;
-#pragma unroll
-        for (int j = 0; j < kEmitPerThread; ++j) {
-            if (fl_gt >> j & 1u) {
-                out[base + gt_before + min(eq_before, need_rem)] = i0 + j;
-                ++gt_before;
-            } else if (fl_eq >> j & 1u) {
-                if (eq_before < need_rem) out[base + gt_before + eq_before] = i0 + j;
-                ++eq_before;
-            }
+        for (int j = 0; j < J; ++j) {
+            const bool g = m_gt >> j & 1u, e = m_eq >> j & 1u;
+            const uint32_t bg = __ballot_sync(0xffffffffu, g), be = __ballot_sync(0xffffffffu, e);
+            const uint32_t gb = gt_before + __popc(bg & lt), eb = eq_before + __popc(be & lt);
+            if (g) out[base + gb + min(eb, need_rem)] = ibase + 32 * j;
+            else if (e && eb < need_rem) out[base + gb + eb] = ibase + 32 * j;
+            gt_before += __popc(bg);
+            eq_before += __popc(be);
         }
-        uint32_t tg = total & 0xffffu, te = min(total >> 16, need_rem);
-        base += tg + te;
+        const uint32_t te = min(total >> 16, need_rem);
+        base += (total & 0xffffu) + te;
         need_rem -= te;
     }
 }

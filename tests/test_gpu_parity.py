@@ -212,7 +212,10 @@ def test_constant_head_contributes_zero():
 def test_select_bit_exact_with_ties():
     """tri_select alone on fp32 scores full of ties: indices must equal the oracle's exactly."""
     g = torch.Generator().manual_seed(5)
-    cases = [(1, 5000, 777, 50), (3, 131072, 4096, 0), (4, 9999, 9998, 7), (2, 4096, 1, 3), (2, 70000, 35000, 1000)]
+    cases = [(1, 5000, 777, 50), (3, 131072, 4096, 0), (4, 9999, 9998, 7), (2, 4096, 1, 3), (2, 70000, 35000, 1000),
+             (1, 32768, 100, 20), (2, 32769, 30000, 0), (1, 500000, 4096, 5000),
+             # very few distinct values: the threshold's value bin overflows the candidate list
+             (1, 50000, 20000, 3), (2, 200000, 4096, 2), (1, 3000, 1500, 1)]
     for U, n, B, levels in cases:
         x = torch.randn(U, n, generator=g)
         if levels:
@@ -229,6 +232,14 @@ def test_select_bit_exact_with_ties():
         for u in range(U):
             want = oracle.select(x[u].double().numpy(), B)
             assert np.array_equal(idx[u].cpu().numpy(), want), (U, n, B, levels, u)
+    # scores far outside the histogram's [-8, 8) range all land in its end bins; the result stays exact
+    x = torch.randn(2, 20000, generator=g) * 1000.0
+    ctx = tb.TriContext(2, 1, 1, torch.zeros(2, 1, 128), torch.zeros(2, 1, 64))
+    idx = torch.full((2, 5000), -1, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(2, dtype=torch.int32, device=DEV)
+    ctx.select(x.to(DEV), torch.tensor([20000], dtype=torch.int32, device=DEV), 20000, 5000, idx, cnt)
+    for u in range(2):
+        assert np.array_equal(idx[u].cpu().numpy(), oracle.select(x[u].double().numpy(), 5000))
     # negative values, -0.0 vs +0.0 and infinities keep the float order
     x = torch.tensor([[0.0, -0.0, -1.0, float("inf"), 1e-40, -1e-40, 3.0, float("-inf")]])
     ctx = tb.TriContext(1, 1, 1, torch.zeros(1, 1, 128), torch.zeros(1, 1, 64))
