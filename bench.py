@@ -76,7 +76,7 @@ class ClockSampler:
         must not fall into a timed region."""
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -269,37 +269,68 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # An in-place round changes its own input (the kept rows move to the front of each sequence's pages), and
+    # a second round on that state would find nearly every kept row already in place.  So for the paged
+    # workload every step starts from the pristine pool: the pages a round overwrites are put back from a copy
+    # between steps, outside the timed region, and each step is timed on its own.
+    restore = None
+    if w.paged:
+        ps = spec.page_size
+        keep_pages = (B + ps - 1) // ps
+        pages = torch.cat([w.page_table[s, :min(keep_pages, (lens[s] + ps - 1) // ps)] for s in range(S)]).long()
+        k_bak, v_bak = w.k[:, pages].clone(), w.v[:, pages].clone()
+
+        def restore():
+            w.k[:, pages] = k_bak
+            w.v[:, pages] = v_bak
+
+    def timed_steps(n):
+        """n steps; returns their total device time in ms (this rank)."""
+        if restore is None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+        evs = []
+        for _ in range(n):
+            restore()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            step()
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in evs)
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     for _ in range(args.warmup):
+        if restore is not None:
+            restore()
         step()
     barrier()
     if args.steps <= 0:
         # fill about one second, so that the clock sampler sees the region under load
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(3):
-            step()
-        e1.record()
+        est = max_over_ranks(timed_steps(3) / 3, dist, dev)
         barrier()
-        est = max_over_ranks(e0.elapsed_time(e1) / 3, dist, dev)
         args.steps = int(min(3000, max(20, 1000.0 / est)))
     sampler.mark()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
+    ms_mine = timed_steps(args.steps)
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms_step = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    ms_step = max_over_ranks(ms_mine, dist, dev) / args.steps
 
     # per-kernel durations: second pass, events recorded by the library between its launches
     ctx.profile_begin()
     per = {k: 0.0 for k in ctx.KERNELS}
     prof_steps = min(args.steps, 200)
     for _ in range(prof_steps):
+        if restore is not None:
+            restore()
         step()
         for k, v in ctx.profile_read().items():
             per[k] += v / prof_steps
@@ -315,7 +346,8 @@ def main():
         "config": {"workload": spec.name + (f"[first {L} layers]" if L != spec.n_layers else ""),
                    "units": U, "layers": L, "kv_heads": H, "group_size": G, "seqs": S, "keys_per_step": keys_per_step,
                    "budget": B, "storage_dtype": "bf16", "paged": bool(w.paged),
-                   "compaction": "in place into the sequence's pages" if w.paged else "out of place",
+                   "compaction": "in place into the sequence's pages, pool restored between steps outside the timed region"
+                   if w.paged else "out of place",
                    "l2": f"inputs larger than L2: {(w.k.numel() + w.v.numel()) * 2 / 1e9:.2f} GB of K+V read per step",
                    "parallelism": "replicas" if world > 1 else "single GPU"},
         "hbm": {"algorithmic_bytes_per_step": abytes, "achieved_gbs": abytes / (ms_step * 1e-3) / 1e9,

@@ -378,8 +378,12 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
     if (aliases(src, dst)) {
         // in place: the prefix whose sources lie inside the destination range goes tile by tile in one block
         // per unit; everything behind it is a hazard-free gather
-        k_compact_inplace<<<U, kInplaceThreads, 0, st>>>(p, rows16 ? 1 : 0);
-        if (rows16) k_gather_rows<true><<<grid, kGatherThreads, 0, st>>>(p);
+        if (rows16) {
+            k_compact_inplace_rows<<<U, kInplaceThreads, 0, st>>>(p);
+            k_gather_rows<true><<<grid, kGatherThreads, 0, st>>>(p);
+        } else {
+            k_compact_inplace_any<<<U, kInplaceThreads, 0, st>>>(p);
+        }
     } else if (rows16) {
         k_gather_rows<false><<<grid, kGatherThreads, 0, st>>>(p);
     } else {

@@ -46,12 +46,12 @@ __device__ __forceinline__ void st_once(void *p, uint4 v)
 // that keeps the kernel at 64 registers, four blocks per SM.
 //
 // AFTER_PREFIX = true is the second phase of an in-place compaction: it moves only the row tiles that
-// k_compact_inplace left alone (tiles whose first source lies at or beyond the kept count), whose sources
-// are all outside the destination range [0, count) -- see k_compact_inplace.
+// k_compact_inplace_rows left alone (tiles whose first source lies at or beyond the kept count), whose sources
+// are all outside the destination range [0, count) -- see k_compact_inplace_rows.
 constexpr int kFastRows = 8;
 constexpr int kFastIters = 2;
 constexpr int kFastRowsPerBlock = kGatherWarps * kFastRows * kFastIters;
-constexpr int kInplaceRows = 32;        // rows per tile of the in-place schedule
+constexpr int kInplaceRows = 128;       // rows per tile of the in-place schedule
 
 template <bool AFTER_PREFIX>
 __global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const CompactParams p)
@@ -168,21 +168,78 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather_any(const CompactPara
 }
 
 // In-place (or aliasing) compaction: one block per unit walks the kept rows in ascending tiles.
-// Every row of a tile is staged in shared memory before any row of the tile is written; since
-// kept_idx[j] >= j and is increasing, a tile's destinations lie strictly below every source of the
-// following tiles, so no source is overwritten before it has been read.  Rows already in their slot
-// (kept_idx[j] == j) are not touched.
+// Every row of a tile is read before any row of the tile is written; since kept_idx[j] >= j and is
+// increasing, a tile's destinations lie strictly below every source of the following tiles, so no source
+// is overwritten before it has been read.  Rows already in their slot (kept_idx[j] == j) are not touched.
 //
-// prefix_only = 1 stops at the first tile whose first source index is >= the kept count: from there on
-// every source lies outside the destination range [0, count), nothing can be overwritten before it is
-// read, and k_gather_rows<true> moves those tiles with full parallelism in a following launch (its
-// destinations, >= the prefix end, are never sources of the prefix, whose sources were all read here first).
+// k_compact_inplace_rows (bf16 K + V): a tile is 128 rows, 8 per warp, held in registers between the loads
+// and the one block barrier that separates them from the stores (lanes and address hand-off as in
+// k_gather_rows).  It stops at the first tile whose first source index is >= the kept count: from there on
+// every source lies outside the destination range [0, count), nothing can be overwritten before it is read,
+// and k_gather_rows<true> moves those tiles with full parallelism in the next launch (its destinations,
+// beyond the prefix, are never sources of the prefix, whose sources were all read here first).
 constexpr int kInplaceThreads = 512;
+static_assert(kInplaceRows == (kInplaceThreads / 32) * kFastRows, "a tile is 8 rows per warp");
 
-__global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace(const CompactParams p, const int prefix_only)
+__global__ void __launch_bounds__(kInplaceThreads, 2) k_compact_inplace_rows(const CompactParams p)
 {
-    __shared__ uint4 stage[kInplaceRows * 48];
-    __shared__ int32_t pos_s[kInplaceRows];
+    const int u = blockIdx.x;
+    const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
+    const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
+    if (threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0) p.new_seq_lens[s] = cnt;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int32_t *idx = p.kept_idx + (int64_t)u * p.budget;
+    const bool is_v = lane >= 16;
+    const char *sb = (is_v ? p.src.v : p.src.k) + (lane & 15) * 16;
+    char *db = (is_v ? p.dst.v : p.dst.k) + (lane & 15) * 16;
+    const int n_src = p.src.n_max;
+
+    for (int t0 = 0; t0 < cnt; t0 += kInplaceRows) {
+        if (__ldg(idx + t0) >= cnt) break;                   // the parallel pass takes over from here
+        const int j0 = t0 + warp * kFastRows;
+        int mine = -1, pos = 0;
+        int64_t so = -1, dof = -1;
+        if (lane < kFastRows && j0 + lane < cnt) {
+            mine = __ldg(idx + j0 + lane);
+            if (mine == j0 + lane) {
+                mine = -1;                                   // already in its slot
+            } else {
+                if (mine >= 0 && mine < n_src) {
+                    so = row_offset(p.src, l, s, h, mine);
+                    dof = row_offset(p.dst, l, s, h, j0 + lane);
+                }
+                if (so < 0 || dof < 0) {
+                    if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
+                    mine = -1; so = -1; dof = -1;
+                } else if (p.dst.positions) {
+                    pos = p.src.positions ? p.src.positions[(int64_t)u * p.src.n_max + mine] : mine;
+                }
+            }
+        }
+        uint4 val[kFastRows];
+#pragma unroll
+        for (int r = 0; r < kFastRows; ++r) {
+            const int64_t o = __shfl_sync(0xffffffffu, so, r);
+            if (o >= 0) val[r] = ld_once(sb + o * 2);
+        }
+        __syncthreads();                                     // every source of the tile has been read
+#pragma unroll
+        for (int r = 0; r < kFastRows; ++r) {
+            const int64_t o = __shfl_sync(0xffffffffu, dof, r);
+            if (o >= 0) *reinterpret_cast<uint4 *>(db + o * 2) = val[r];
+        }
+        if (p.dst.positions && mine >= 0) p.dst.positions[(int64_t)u * p.dst.n_max + j0 + lane] = pos;
+    }
+}
+
+// The same schedule for the remaining cases (fp32 keys, no value cache): 32-row tiles staged in shared
+// memory, the whole unit in one block.
+constexpr int kInplaceAnyRows = 32;
+
+__global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace_any(const CompactParams p)
+{
+    __shared__ uint4 stage[kInplaceAnyRows * 48];
+    __shared__ int32_t pos_s[kInplaceAnyRows];
     const int u = blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
@@ -190,9 +247,8 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace(const Compa
     const int32_t *idx = p.kept_idx + (int64_t)u * p.budget;
     const int per_row = p.k_vec + p.v_vec;
 
-    for (int j0 = 0; j0 < cnt; j0 += kInplaceRows) {
-        if (prefix_only && __ldg(idx + j0) >= cnt) break;
-        const int rows = min(kInplaceRows, cnt - j0);
+    for (int j0 = 0; j0 < cnt; j0 += kInplaceAnyRows) {
+        const int rows = min(kInplaceAnyRows, cnt - j0);
         for (int i = threadIdx.x; i < rows * per_row; i += kInplaceThreads) {
             int r = i / per_row, c = i - r * per_row;
             int srow = __ldg(idx + j0 + r);

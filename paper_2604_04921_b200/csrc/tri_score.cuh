@@ -44,26 +44,12 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ void mma_tf32_1688(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                              uint32_t a3, uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};\n"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 __device__ __forceinline__ float fast_sqrt(float x)
 {
     float r;
     asm("sqrt.approx.ftz.f32 %0, %1;\n" : "=f"(r) : "f"(x));
     return r;
 }
-
-// Upper part of an fp32 that is exactly representable in tf32 (10 explicit mantissa bits).  With
-// lo = x - hi (exact), hi + lo carries x to ~2^-22 through two tf32 MMAs.
-__device__ __forceinline__ uint32_t to_tf32(float x) { return __float_as_uint(x) & 0xffffe000u; }
 
 // Packed fp32 pairs (sm_100 f32x2 arithmetic): two lanes per instruction.
 __device__ __forceinline__ uint64_t pack2(float a, float b)
@@ -225,6 +211,10 @@ __device__ __forceinline__ float zmax4(float4 x, const float *mu_s, const float 
     return fmaxf(fmaxf((x.x - mu_s[0]) * rs_s[0], (x.y - mu_s[1]) * rs_s[1]),
                  fmaxf((x.z - mu_s[2]) * rs_s[2], (x.w - mu_s[3]) * rs_s[3]));
 }
+__device__ __forceinline__ float zmax8(const float4 *row, const float *mu_s, const float *rs_s)
+{
+    return fmaxf(zmax4(row[0], mu_s, rs_s), zmax4(row[1], mu_s + 4, rs_s + 4));
+}
 __device__ __forceinline__ float zmax(const float *row, int G, const float *mu_s, const float *rs_s)
 {
     float z = -INFINITY;
@@ -264,6 +254,9 @@ __global__ void __launch_bounds__(256) k_normalize(const NormParams p)
     if (G == 4) {
         for (int key = key_begin + tid; key < key_end; key += 256)
             out[key] = zmax4(*reinterpret_cast<const float4 *>(rawu + (int64_t)key * 4), mu_s, rs_s);
+    } else if (G == 8) {
+        for (int key = key_begin + tid; key < key_end; key += 256)
+            out[key] = zmax8(reinterpret_cast<const float4 *>(rawu + (int64_t)key * 8), mu_s, rs_s);
     } else {
         for (int key = key_begin + tid; key < key_end; key += 256)
             out[key] = zmax(rawu + (int64_t)key * G, G, mu_s, rs_s);

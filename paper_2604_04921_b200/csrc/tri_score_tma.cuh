@@ -10,8 +10,9 @@
 //
 // Arithmetic per k-step s (dims 16s..16s+15 of 16 keys):
 //   trig   one bf16 MMA of the fragment with the (hi, lo)-split W              (Sections 4.1, 4.2)
-//   norm   the fragment's four registers are four (re, im) pairs = four bands; their magnitudes,
-//          split hi + lo for tf32, are the A fragment of two m16n8k8 tf32 MMAs with m_f (Section 4.2)
+//   norm   the fragment's four registers are four (re, im) pairs = four bands; the eight magnitudes of two
+//          k-steps, split into a bf16 value and a bf16 residual, are the A fragments of two more bf16 MMAs
+//          against m_f, itself split the same way into two columns per head           (Section 4.2)
 // both accumulate into the same fp32 accumulator: thread (q, t) ends with S~ of head 4nt + t for keys
 // q and q+8 of the tile.
 #pragma once
@@ -73,33 +74,36 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
                  : "memory");
 }
 
-// |(re_a, im_a)| and |(re_b, im_b)| split for tf32: hi as tf32 bit patterns, lo the exact remainders.
-__device__ __forceinline__ void mags2(float re_a, float im_a, float re_b, float im_b, uint32_t &hi_a,
-                                      uint32_t &hi_b, uint32_t &lo_a, uint32_t &lo_b)
-{
-    uint64_t re = pack2(re_a, re_b), im = pack2(im_a, im_b);
-    float sa, sb;
-    unpack2(fma2(re, re, mul2(im, im)), sa, sb);
-    float ma = fast_sqrt(sa), mb = fast_sqrt(sb);
-    hi_a = to_tf32(ma);
-    hi_b = to_tf32(mb);
-    float la, lb;
-    unpack2(sub2(pack2(ma, mb), pack2(__uint_as_float(hi_a), __uint_as_float(hi_b))), la, lb);
-    lo_a = __float_as_uint(la);
-    lo_b = __float_as_uint(lb);
-}
 __device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t cvt_bf16x2(float upper, float lower)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(upper), "f"(lower));
+    return r;
+}
+// |(re0, im0)| and |(re1, im1)| as a packed bf16 pair `hi` (first magnitude in the lower half) and the bf16
+// pair `lo` of what the rounding left over: hi + lo carries each magnitude to ~2^-17.
+__device__ __forceinline__ void mag_pair(float re0, float im0, float re1, float im1, uint32_t &hi, uint32_t &lo)
+{
+    uint64_t re = pack2(re0, re1), im = pack2(im0, im1);
+    float s0, s1;
+    unpack2(fma2(re, re, mul2(im, im)), s0, s1);
+    const float m0 = fast_sqrt(s0), m1 = fast_sqrt(s1);
+    hi = cvt_bf16x2(m1, m0);
+    float r0, r1;
+    unpack2(sub2(pack2(m0, m1), pack2(bf16_lo(hi), bf16_hi(hi))), r0, r1);
+    lo = cvt_bf16x2(r1, r0);
+}
 
 template <int NT, int LAYOUT>
 __global__ void __launch_bounds__(kScoreThreads, 3)
 k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
 {
     extern __shared__ __align__(1024) uint8_t tiles[];   // [warp][stage][half][16 rows][128 B]
-    __shared__ float Wf[NT * 4][kHeadDim];
-    __shared__ float Mf[NT * 4][kBands];
     __shared__ uint2 trigB[NT][8][32];
-    __shared__ uint2 normB[NT][8][32];
+    __shared__ uint2 normB[NT][4][32];
     __shared__ double red[kScoreWarps][NT * 4][2];
     __shared__ __align__(8) uint64_t bars[kScoreWarps][kStages];
 
@@ -144,45 +148,47 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
         for (int it = 0; it < kStages && it < my_n; ++it) issue(it);
     }
 
-    // ---- fold, step 2 (overlaps the first loads): W_f^(g) = E[q_f]^(g) * E[s][f], split for the MMAs ----
-    for (int i = tid; i < NT * 4 * kBands; i += kScoreThreads) {
-        int g = i / kBands, f = i - g * kBands;
-        int ir = LAYOUT == 0 ? 2 * f : f, ii = LAYOUT == 0 ? 2 * f + 1 : f + kBands;
-        float wr = 0.f, wi = 0.f, m = 0.f;
-        if (g < G) {
-            const float *c = p.qc + ((int64_t)l * p.H * G + (int64_t)h * G + g) * kHeadDim;
-            double cr = c[ir], ci = c[ii];
-            double2 e = p.E[s * kBands + f];
-            wr = (float)(cr * e.x - ci * e.y);
-            wi = (float)(cr * e.y + ci * e.x);
-            m = p.mw[((int64_t)l * p.H * G + (int64_t)h * G + g) * kBands + f];
-        }
-        Wf[g][ir] = wr;
-        Wf[g][ii] = wi;
-        Mf[g][f] = m;
-    }
-    __syncthreads();
+    // ---- fold, step 2 (overlaps the first loads): W_f^(g) = E[q_f]^(g) * E[s][f], straight into the B fragments
+    // of the MMAs, each value split into a bf16 and the bf16 of its residual (two columns per head) ----
     for (int i = tid; i < NT * 8 * 32; i += kScoreThreads) {
-        int ln = i & 31, st = (i >> 5) & 7, nt = i >> 8;
-        int col = ln >> 2, t = ln & 3;          // B fragment: column = lane/4, k slots from lane%4
-        int g = 4 * nt + (col >> 1), part = col & 1;
-        uint32_t w[4];
+        const int ln = i & 31, st = (i >> 5) & 7, nt = i >> 8;
+        const int col = ln >> 2, t = ln & 3;          // B fragment: column = lane/4, k slots from lane%4
+        const int g = 4 * nt + (col >> 1), part = col & 1;
+        const int64_t qh = (int64_t)l * p.H * G + (int64_t)h * G + g;
+        const float *c = p.qc + qh * kHeadDim;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        if (g < G) {
 #pragma unroll
-        for (int x = 0; x < 4; ++x) {            // k slots 2t, 2t+1, 2t+8, 2t+9 of step st
-            float v = Wf[g][16 * st + 2 * t + (x & 1) + 8 * (x >> 1)];
-            uint32_t hi = bf16_hi_bits(v);
-            w[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+            for (int x = 0; x < 4; ++x) {            // k slots 2t, 2t+1, 2t+8, 2t+9 of step st = dims of the key row
+                const int d = 16 * st + 2 * t + (x & 1) + 8 * (x >> 1);
+                const int f = LAYOUT == 0 ? d >> 1 : d & (kBands - 1);
+                const bool imag = LAYOUT == 0 ? (d & 1) : (d >= kBands);
+                const int ir = LAYOUT == 0 ? 2 * f : f, ii = LAYOUT == 0 ? 2 * f + 1 : f + kBands;
+                const double cr = c[ir], ci = c[ii];
+                const double2 e = p.E[s * kBands + f];
+                const float v = imag ? (float)(cr * e.y + ci * e.x) : (float)(cr * e.x - ci * e.y);
+                const uint32_t hi = bf16_hi_bits(v);
+                w[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+            }
         }
         trigB[nt][st][ln] = make_uint2(w[0] | (w[1] << 16), w[2] | (w[3] << 16));
-        // norm: tf32 step st, k slot t and t+4
-        int b0, b1;
-        if (LAYOUT == 0) { b0 = 8 * st + t; b1 = 8 * st + 4 + t; }
-        else { int ss = st >> 1, hf = st & 1; b0 = 16 * ss + 2 * t + hf; b1 = 16 * ss + 8 + 2 * t + hf; }
-        float m0 = Mf[g][b0], m1 = Mf[g][b1];
-        uint32_t h0 = to_tf32(m0), h1 = to_tf32(m1);
-        normB[nt][st][ln] = part == 0 ? make_uint2(h0, h1)
-                                      : make_uint2(__float_as_uint(m0 - __uint_as_float(h0)),
-                                                   __float_as_uint(m1 - __uint_as_float(h1)));
+        // norm: B fragment of pair st < 4 (k-steps 2 st and 2 st + 1 of the keys): k slots 2t, 2t+1, 2t+8, 2t+9
+        // stand for the bands whose magnitudes the main loop puts there
+        if (st < 4) {
+            int bnd[4];
+            if (LAYOUT == 0) { bnd[0] = 16 * st + t; bnd[1] = 16 * st + 4 + t; bnd[2] = 16 * st + 8 + t; bnd[3] = 16 * st + 12 + t; }
+            else { bnd[0] = 16 * st + 2 * t; bnd[1] = bnd[0] + 1; bnd[2] = 16 * st + 8 + 2 * t; bnd[3] = bnd[2] + 1; }
+            uint32_t m[4] = {0u, 0u, 0u, 0u};
+            if (g < G) {
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    const float v = p.mw[qh * kBands + bnd[x]];
+                    const uint32_t hi = bf16_hi_bits(v);
+                    m[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+                }
+            }
+            normB[nt][st][ln] = make_uint2(m[0] | (m[1] << 16), m[2] | (m[3] << 16));
+        }
     }
     __syncthreads();
 
@@ -223,40 +229,26 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
                 mma_bf16_16816(acc[nt], X[st][0], X[st][1], X[st][2], X[st][3], b.x, b.y);
             }
         }
-        if (LAYOUT == 0) {
 #pragma unroll
-            for (int st = 0; st < 8; ++st) {
-                uint32_t hA[4], lA[4];
-                mags2(bf16_lo(X[st][0]), bf16_hi(X[st][0]), bf16_lo(X[st][1]), bf16_hi(X[st][1]), hA[0], hA[1], lA[0], lA[1]);
-                mags2(bf16_lo(X[st][2]), bf16_hi(X[st][2]), bf16_lo(X[st][3]), bf16_hi(X[st][3]), hA[2], hA[3], lA[2], lA[3]);
+        for (int pr = 0; pr < 4; ++pr) {
+            uint32_t hA[4], lA[4];
+            if (LAYOUT == 0) {
+                const uint32_t *a = X[2 * pr], *b = X[2 * pr + 1];      // one register = (re, im) of one band
+                mag_pair(bf16_lo(a[0]), bf16_hi(a[0]), bf16_lo(a[2]), bf16_hi(a[2]), hA[0], lA[0]);
+                mag_pair(bf16_lo(a[1]), bf16_hi(a[1]), bf16_lo(a[3]), bf16_hi(a[3]), hA[1], lA[1]);
+                mag_pair(bf16_lo(b[0]), bf16_hi(b[0]), bf16_lo(b[2]), bf16_hi(b[2]), hA[2], lA[2]);
+                mag_pair(bf16_lo(b[1]), bf16_hi(b[1]), bf16_lo(b[3]), bf16_hi(b[3]), hA[3], lA[3]);
+            } else {
+                const uint32_t *re = X[pr], *im = X[pr + 4];            // two bands per register, re and im apart
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    uint2 b = normB[nt][st][lane];
-                    mma_tf32_1688(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
-                    mma_tf32_1688(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
-                }
+                for (int x = 0; x < 4; ++x)
+                    mag_pair(bf16_lo(re[x]), bf16_lo(im[x]), bf16_hi(re[x]), bf16_hi(im[x]), hA[x], lA[x]);
             }
-        } else {
 #pragma unroll
-            for (int ss = 0; ss < 4; ++ss) {
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    uint32_t hA[4], lA[4];
-                    const uint32_t *re = X[ss], *im = X[ss + 4];
-                    if (hf == 0) {
-                        mags2(bf16_lo(re[0]), bf16_lo(im[0]), bf16_lo(re[1]), bf16_lo(im[1]), hA[0], hA[1], lA[0], lA[1]);
-                        mags2(bf16_lo(re[2]), bf16_lo(im[2]), bf16_lo(re[3]), bf16_lo(im[3]), hA[2], hA[3], lA[2], lA[3]);
-                    } else {
-                        mags2(bf16_hi(re[0]), bf16_hi(im[0]), bf16_hi(re[1]), bf16_hi(im[1]), hA[0], hA[1], lA[0], lA[1]);
-                        mags2(bf16_hi(re[2]), bf16_hi(im[2]), bf16_hi(re[3]), bf16_hi(im[3]), hA[2], hA[3], lA[2], lA[3]);
-                    }
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        uint2 b = normB[nt][2 * ss + hf][lane];
-                        mma_tf32_1688(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
-                        mma_tf32_1688(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
-                    }
-                }
+            for (int nt = 0; nt < NT; ++nt) {
+                const uint2 b = normB[nt][pr][lane];
+                mma_bf16_16816(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
+                mma_bf16_16816(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
             }
         }
 

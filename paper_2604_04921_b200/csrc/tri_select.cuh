@@ -140,6 +140,13 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
                 scw[i] = z;
                 atomicAdd(&hist[value_bin(z)], 1u);
             }
+        } else if (p.G == 8) {
+#pragma unroll 4
+            for (int i = tid; i < n; i += kSelThreads) {
+                const float z = zmax8(reinterpret_cast<const float4 *>(rawu + (int64_t)i * 8), mu_s, rs_s);
+                scw[i] = z;
+                atomicAdd(&hist[value_bin(z)], 1u);
+            }
         } else {
             for (int i = tid; i < n; i += kSelThreads) {
                 const float z = zmax(rawu + (int64_t)i * p.G, p.G, mu_s, rs_s);
