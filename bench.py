@@ -36,11 +36,11 @@ NOMINAL_HBM_GBS = 8000.0
 
 
 # DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum on
-# 1,048,576 keys: 268.564736 MB + 13.445376 MB), valid only for the kernel source it was taken on.
-SCORE_TRAFFIC = {"bytes_per_key": (268564736 + 13445376) / 1048576,
+# 1,048,576 keys: 268.562688 MB + 15.030272 MB), valid only for the kernel source it was taken on.
+SCORE_TRAFFIC = {"bytes_per_key": (268562688 + 15030272) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
-                 "sha256": "1fae8a5229be2e5184832882617f8c1545fe0a1908945553fad8315c9ca44fb0"}
+                 "sha256": "4efb7ee835935b415f830b6806653bfb423a1bdda6a7f99d62bb19dda332cf05"}
 
 
 def score_traffic_per_launch(keys):
@@ -384,6 +384,7 @@ def main():
 
         step_host()
         barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(e2e_steps):
             step_host()

@@ -317,3 +317,53 @@ def test_full_size_config1_sampled_units():
     for (l, h) in [(0, 0), (35, 7)]:
         ref = oracle_unit(w, l, 0, h, sp.budget)
         check_unit(w, res, ref, l, 0, h, sp.budget)
+
+
+def _whole_job_invariants(w, res, budget):
+    """Properties that hold at any size: counts, strictly ascending in-range indices."""
+    sp = w.spec
+    assert int(res["status"].item()) == 0
+    lens = w.seq_lens.repeat_interleave(sp.n_kv_heads).repeat(w.k.shape[0])
+    want = torch.clamp(lens, max=budget)
+    assert torch.equal(res["kept_cnt"], want)
+    idx = res["kept_idx"]
+    col = torch.arange(budget, device=idx.device)[None, :]
+    valid = col < want[:, None]
+    assert torch.all((idx >= 0) | ~valid) and torch.all((idx < lens[:, None]) | ~valid)
+    assert torch.all((idx[:, 1:] > idx[:, :-1]) | ~valid[:, 1:])
+
+
+def test_full_size_config2_sampled_units():
+    """The steady-state batch at full size (36 x 64 x 8 units of 2,176 keys at scattered positions)."""
+    sp = W.SPECS["qwen3_8b_steady_b64"]
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget, want_scores=False)
+    _whole_job_invariants(w, res, sp.budget)
+    assert res["new_seq_lens"].tolist() == [sp.budget] * sp.n_seqs
+    for (l, s, h) in [(0, 0, 0), (17, 33, 5), (35, 63, 7)]:
+        check_unit(w, res, oracle_unit(w, l, s, h, sp.budget), l, s, h, sp.budget)
+
+
+def test_full_size_config3_sampled_units():
+    """The 131,072-token sequence at full size (36 x 8 units), mixed per-head noise."""
+    sp = W.SPECS["qwen3_8b_long_128k"]
+    w = W.make_workload(sp, DEV)
+    res = run_compress(w, sp.budget, want_scores=False)
+    _whole_job_invariants(w, res, sp.budget)
+    for (l, h) in [(0, 0), (35, 7)]:
+        check_unit(w, res, oracle_unit(w, l, 0, h, sp.budget), l, 0, h, sp.budget)
+
+
+def test_full_size_config4_slab_sampled_units():
+    """The ragged paged batch at full size per layer (16 sequences of 8K-64K keys, G = 8), a slab of 4 of
+    its 64 layers as the benchmark runs it, compacted in place into the sequences' own pages."""
+    sp = W.SPECS["qwen3_32b_ragged_paged"]
+    w = W.make_workload(sp, DEV, layer0=0, n_layers=4)
+    lens = w.seq_lens.tolist()
+    picks = [(0, lens.index(min(lens)), 0), (3, lens.index(max(lens)), 7)]
+    refs = {u: oracle_unit(w, *u, sp.budget) for u in picks}      # before the in-place write
+    res = run_compress(w, sp.budget, in_place=True, want_scores=False)
+    _whole_job_invariants(w, res, sp.budget)
+    assert res["new_seq_lens"].tolist() == [min(n, sp.budget) for n in lens]
+    for u, ref in refs.items():
+        check_unit(w, res, ref, *u, sp.budget)
