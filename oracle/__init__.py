@@ -61,6 +61,8 @@ def _load():
     lib.tri_oracle_unit_bf16.argtypes = [P, P, c_i64, c_i, c_i64, P, P, c_i, P, c_i, c_d, c_i, c_i,
                                          c_i64, P, P, P]
     lib.tri_oracle_unit_bf16.restype = c_i64
+    lib.tri_oracle_calibrate.argtypes = [P, c_i64, c_i, c_i, P, P, P]
+    lib.tri_oracle_calibrate.restype = None
     lib.tri_oracle_num_threads.argtypes = []
     lib.tri_oracle_num_threads.restype = c_i
     _lib = lib
@@ -182,3 +184,15 @@ def unit_bf16(k_post_bits, pos, p_q: int, q_center, q_mean_norm, B: int, offsets
                                        int(layout), int(norm_variant), int(B), _p(raw), _p(s), _p(idx))
     assert cnt == idx.size
     return raw, s, idx
+
+
+def calibrate(q, layout: int = 0):
+    """Calibration statistics of one query head from its pre-RoPE queries q[T, d]:
+    returns (center[d], mean_norm[d/2], mrl[d/2]) = (E[q_f], E|q_f|, R_f)."""
+    q = _f64(q)
+    T, d = q.shape
+    center = np.empty(d, dtype=np.float64)
+    mean_norm = np.empty(d // 2, dtype=np.float64)
+    mrl = np.empty(d // 2, dtype=np.float64)
+    _load().tri_oracle_calibrate(_p(q), T, d, int(layout), _p(center), _p(mean_norm), _p(mrl))
+    return center, mean_norm, mrl

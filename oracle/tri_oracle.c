@@ -274,3 +274,32 @@ int tri_oracle_num_threads(void)
     return 1;
 #endif
 }
+
+/* ---- calibration statistics (Sections 3.3, 4.1, Appendix B.5) ----------------------- */
+
+/*
+ * Per band f over T pre-RoPE query vectors q[t]:
+ *   center      E[q_f]   complex mean, stored in the input's own component layout   [d]
+ *   mean_norm   E|q_f|   mean of the band magnitudes                                 [d/2]
+ *   mrl         R_f = |E[q_f]| / E|q_f|  (mean resultant length; 0 where E|q_f| = 0) [d/2]
+ * Plain sums in double, token by token.
+ */
+void tri_oracle_calibrate(const double *q, int64_t T, int d, int layout, double *center,
+                          double *mean_norm, double *mrl)
+{
+    const int F = d / 2;
+    for (int i = 0; i < d; ++i) center[i] = 0.0;
+    for (int f = 0; f < F; ++f) mean_norm[f] = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        const double *x = q + t * d;
+        for (int i = 0; i < d; ++i) center[i] += x[i];
+        for (int f = 0; f < F; ++f)
+            mean_norm[f] += hypot(x[re_index(f, F, layout)], x[im_index(f, F, layout)]);
+    }
+    for (int i = 0; i < d; ++i) center[i] /= (double)T;
+    for (int f = 0; f < F; ++f) {
+        mean_norm[f] /= (double)T;
+        double cn = hypot(center[re_index(f, F, layout)], center[im_index(f, F, layout)]);
+        mrl[f] = mean_norm[f] > 0.0 ? cn / mean_norm[f] : 0.0;
+    }
+}

@@ -149,20 +149,31 @@ def _head_noise(spec: Spec, device) -> torch.Tensor:
     return spec.noise_lo + (spec.noise_hi - spec.noise_lo) * u
 
 
+def make_queries(spec: Spec, layer: int, n_tokens: int, device="cpu", dtype=torch.float64) -> torch.Tensor:
+    """Pre-RoPE calibration queries of one layer: q = c_q + s * eps per query head, [n_tokens, Hq, 128].
+    The draws come in blocks of N_CALIB tokens, so the first N_CALIB tokens do not depend on n_tokens."""
+    H, G = spec.n_kv_heads, spec.group_size
+    noise = _head_noise(spec, "cpu")
+    g = _gen(device, spec.name, "q", layer)
+    centre = torch.randn(H * G, 1, HEAD_DIM, generator=g, dtype=torch.float64, device=device)
+    std = noise[layer].repeat_interleave(G).view(H * G, 1, 1).to(device)
+    out = torch.empty(n_tokens, H * G, HEAD_DIM, dtype=dtype, device=device)
+    for t0 in range(0, n_tokens, N_CALIB):
+        eps = torch.randn(H * G, N_CALIB, HEAD_DIM, generator=g, dtype=torch.float64, device=device)
+        n = min(N_CALIB, n_tokens - t0)
+        out[t0:t0 + n] = (centre + std * eps)[:, :n].transpose(0, 1).to(dtype)
+    return out
+
+
 def make_stats(spec: Spec):
     """Calibration statistics per query head as sample means over N_CALIB seeded draws
     q = c_q + eps (Section 3.3 / 4.1: E[q_f] and E|q_f| come from calibration data).
     Returns q_center [L, Hq, 128] fp32 and q_mean_norm [L, Hq, 64] fp32 on the host."""
     L, H, G = spec.n_layers, spec.n_kv_heads, spec.group_size
-    noise = _head_noise(spec, "cpu")
     qc = torch.empty(L, H * G, HEAD_DIM, dtype=torch.float32)
     qn = torch.empty(L, H * G, HEAD_DIM // 2, dtype=torch.float32)
     for l in range(L):
-        g = _gen("cpu", spec.name, "q", l)
-        centre = torch.randn(H * G, 1, HEAD_DIM, generator=g, dtype=torch.float64)
-        eps = torch.randn(H * G, N_CALIB, HEAD_DIM, generator=g, dtype=torch.float64)
-        std = noise[l].repeat_interleave(G).view(H * G, 1, 1)
-        q = centre + std * eps
+        q = make_queries(spec, l, N_CALIB, "cpu").transpose(0, 1)          # [Hq, N_CALIB, 128] float64
         qc[l] = q.mean(dim=1).to(torch.float32)
         qn[l] = torch.sqrt(q[..., 0::2] ** 2 + q[..., 1::2] ** 2).mean(dim=1).to(torch.float32)
     return qc, qn

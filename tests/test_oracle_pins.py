@@ -309,3 +309,48 @@ def test_unit_bf16_chains_the_steps(rng):
     _, s2 = oracle.normalize(raw2)
     assert np.array_equal(s, s2)
     assert np.array_equal(idx, oracle.select(s2, B))
+
+
+def test_calibration_statistics_pins(rng):
+    """E[q_f], E|q_f| and R_f against closed forms and an independent computation."""
+    T = 360
+    # identical vectors: centre = the vector, mean norm = its band magnitudes, R = 1 in every band
+    v = rng.standard_normal(D)
+    c, n, r = oracle.calibrate(np.tile(v, (T, 1)))
+    assert np.allclose(c, v, rtol=1e-13) and np.allclose(n, band_abs(v), rtol=1e-13) and np.allclose(r, 1.0, rtol=1e-12)
+    # band f turning through whole circles at constant radius: centre 0, mean norm = radius, R = 0
+    q = np.zeros((T, D))
+    ang = 2 * math.pi * np.arange(T) / T
+    for f in range(F):
+        q[:, 2 * f], q[:, 2 * f + 1] = (f + 1) * np.cos((f % 5 + 1) * ang), (f + 1) * np.sin((f % 5 + 1) * ang)
+    c, n, r = oracle.calibrate(q)
+    assert np.max(np.abs(c)) < 1e-12 and np.allclose(n, np.arange(1, F + 1), rtol=1e-13) and np.max(r) < 1e-12
+    # two opposite phases with weights 3:1 at unit radius: R = |3 - 1| / 4 = 1/2
+    q = np.zeros((4, D)); q[:3, 10] = 1.0; q[3, 10] = -1.0
+    c, n, r = oracle.calibrate(q)
+    assert c[10] == pytest.approx(0.5) and n[5] == pytest.approx(1.0) and r[5] == pytest.approx(0.5)
+    assert r[0] == 0.0                                   # an all-zero band: R defined as 0
+    # random data: numpy on complex numbers, 0 <= R <= 1 (Appendix B.5), and the half-split layout as a permutation
+    q = rng.standard_normal((T, D)) * 0.5 + rng.standard_normal(D)
+    c, n, r = oracle.calibrate(q)
+    z = q[:, 0::2] + 1j * q[:, 1::2]
+    assert np.allclose(c[0::2] + 1j * c[1::2], z.mean(axis=0), rtol=1e-12)
+    assert np.allclose(n, np.abs(z).mean(axis=0), rtol=1e-12)
+    assert np.allclose(r, np.abs(z.mean(axis=0)) / np.abs(z).mean(axis=0), rtol=1e-12)
+    assert np.all(r >= 0.0) and np.all(r <= 1.0 + 1e-15)
+    perm = np.concatenate([np.arange(0, D, 2), np.arange(1, D, 2)])
+    c2, n2, r2 = oracle.calibrate(q[:, perm], layout=1)
+    assert np.allclose(c2, c[perm], rtol=1e-13) and np.allclose(n2, n, rtol=1e-13) and np.allclose(r2, r, rtol=1e-12)
+
+
+def test_calibration_matches_the_workload_generator_statistics():
+    """The input generator computes its per-head statistics with torch; the oracle must agree on the same draws."""
+    import torch
+    from paper_2604_04921_b200 import workloads as W
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="calibpin", n_layers=1, n_kv_heads=1, group_size=2)
+    q = W.make_queries(sp, 0, W.N_CALIB, "cpu", dtype=torch.float64)          # [T, Hq, 128]
+    qc, qn = W.make_stats(sp)
+    for hq in range(2):
+        c, n, r = oracle.calibrate(q[:, hq].numpy())
+        assert np.allclose(c, qc[0, hq].double().numpy(), atol=1e-6)
+        assert np.allclose(n, qn[0, hq].double().numpy(), atol=1e-6)
