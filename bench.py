@@ -203,6 +203,54 @@ def run_reference(args, spec):
     print(json.dumps(line), flush=True)
 
 
+def run_calibration(args):
+    """--calibration: the statistics pass that feeds the round (E[q_f], E|q_f|, R_f of one layer's query heads
+    from bf16 pre-RoPE queries), on a Qwen3-8B-shaped layer: 32 heads x 262,144 tokens (the calibration sets of
+    the paper's sensitivity study hold 50k to 960k tokens).  One step = one pass over the layer's queries."""
+    import torch
+    from paper_2604_04921_b200 import binding as tb
+    from paper_2604_04921_b200 import workloads as W
+    torch.cuda.set_device(0)
+    tb.lib()
+    sp = W.SPECS["qwen3_8b_oneshot_32k"]
+    T, Hq = 262144, sp.n_kv_heads * sp.group_size
+    q = W.make_queries(sp, 0, T, "cuda", dtype=torch.bfloat16)
+    cal = tb.Calibrator(Hq)
+    for _ in range(max(3, args.warmup)):
+        cal.add(q)
+    torch.cuda.synchronize()
+    steps = args.steps if args.steps > 0 else 1000
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        cal.add(q)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    peak, peak_src = measured_peaks()
+    nbytes = q.numel() * 2
+    line = {"metric": "tri_calib_accumulate query rows (token x head) per sec", "value": T * Hq / (ms * 1e-3), "unit": "rows/s",
+            "n_gpus": 1, "steps": steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "calibration qwen3_8b layer", "tokens": T, "heads": Hq, "storage_dtype": "bf16",
+                       "l2": f"inputs larger than L2: {nbytes / 1e9:.2f} GB read per step"},
+            "roofline": {"kernel": "k_calib_partial (+ k_calib_merge)", "bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9,
+                         "peak": peak, "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / peak, "traffic": None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": nbytes},
+            "gpu_launches": 2 * steps}
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        qs = q[:16384, :4].double().cpu().numpy()
+        t0 = time.perf_counter()
+        for h in range(4):
+            oracle.calibrate(qs[:, h])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": 16384 * 4 / dt, "unit": "rows/s", "cores": 1, "kind": "oracle",
+                                "sample": "16,384 tokens x 4 heads"}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -213,7 +261,11 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (a slab); 0 = all")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--calibration", action="store_true", help="time the calibration-statistics pass instead of the round")
     args = ap.parse_args()
+    if args.calibration:
+        run_calibration(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
     from paper_2604_04921_b200 import workloads as W

@@ -207,6 +207,30 @@ tri_status tri_profile_begin(tri_ctx *ctx);
 tri_status tri_profile_read(tri_ctx *ctx, float *ms);
 tri_status tri_profile_end(tri_ctx *ctx);
 
+/*
+ * Calibration statistics (Section 4.1: "computed from calibration data"; Section 3.3; Appendix B.5).
+ * For one layer's query heads, from pre-RoPE query vectors of calibration tokens:
+ *   E[q_f]   complex mean per band              -> q_center    [n_heads][128] fp32, in the input's component layout
+ *   E|q_f|   mean band magnitude                -> q_mean_norm [n_heads][64]  fp32
+ *   R_f = |E[q_f]| / E|q_f|  (mean resultant length, 0 where E|q_f| = 0)  -> mrl [n_heads][64] fp32, may be NULL
+ * which are exactly the two arrays tri_create takes.  The statistics are streamed: tri_calib_reset zeroes a
+ * running state, tri_calib_accumulate adds T more tokens (call it once per chunk of the calibration set),
+ * tri_calib_finalize turns the state into means.  All device pointers; all calls asynchronous on `stream`.
+ *   state   device, tri_calib_state_bytes(n_heads) bytes, 8-byte aligned: fp64 sums and the token count
+ *   q       device [T][n_heads][128]: bf16 (q_kind 0) or fp32 (q_kind 1); stride_tok / stride_head in elements,
+ *           multiples of 4 (q_kind 0: 8-byte rows) resp. 4 (q_kind 1: 16-byte rows); q aligned likewise
+ *   ws      device scratch of tri_calib_workspace_bytes(n_heads, T) bytes, 8-byte aligned
+ * Sums are formed in a fixed order (no atomics), so equal inputs give equal bits.
+ */
+size_t     tri_calib_state_bytes(int32_t n_heads);
+size_t     tri_calib_workspace_bytes(int32_t n_heads, int64_t T);
+tri_status tri_calib_reset(void *state, int32_t n_heads, void *stream);
+tri_status tri_calib_accumulate(const void *q, int32_t q_kind, int64_t T, int32_t n_heads, int64_t stride_tok,
+                                int64_t stride_head, int32_t pair_layout, void *state, void *ws, size_t ws_bytes,
+                                void *stream);
+tri_status tri_calib_finalize(const void *state, int32_t n_heads, int32_t pair_layout, float *q_center,
+                              float *q_mean_norm, float *mrl, void *stream);
+
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char *tri_last_cuda_error(void);
 

@@ -20,12 +20,14 @@ _ROOT = _PKG.parent
 LIB_PATH = _PKG / "lib" / "libtriattn.so"
 SOURCES = [_PKG / "csrc" / "tri_api.cu"]
 HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cuh", _PKG / "csrc" / "tri_score.cuh",
-           _PKG / "csrc" / "tri_score_tma.cuh",
+           _PKG / "csrc" / "tri_score_tma.cuh", _PKG / "csrc" / "tri_calib.cuh",
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",
            "tri_compress", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_last_cuda_error",
-           "tri_profile_begin", "tri_profile_read", "tri_profile_end"]
+           "tri_profile_begin", "tri_profile_read", "tri_profile_end",
+           "tri_calib_state_bytes", "tri_calib_workspace_bytes", "tri_calib_reset", "tri_calib_accumulate",
+           "tri_calib_finalize"]
 
 STATUS = {0: "TRI_OK", 1: "TRI_ERR_INVALID_ARG", 2: "TRI_ERR_UNSUPPORTED", 3: "TRI_ERR_WORKSPACE",
           4: "TRI_ERR_CUDA", 5: "TRI_ERR_DEVICE_CHECK"}
@@ -110,6 +112,17 @@ def lib():
         fn.restype = ctypes.c_int
     L.tri_profile_read.argtypes = [P, P]
     L.tri_profile_read.restype = ctypes.c_int
+    i64 = ctypes.c_int64
+    L.tri_calib_state_bytes.argtypes = [i32]
+    L.tri_calib_state_bytes.restype = sz
+    L.tri_calib_workspace_bytes.argtypes = [i32, i64]
+    L.tri_calib_workspace_bytes.restype = sz
+    L.tri_calib_reset.argtypes = [P, i32, P]
+    L.tri_calib_reset.restype = ctypes.c_int
+    L.tri_calib_accumulate.argtypes = [P, i32, i64, i32, i64, i64, i32, P, P, sz, P]
+    L.tri_calib_accumulate.restype = ctypes.c_int
+    L.tri_calib_finalize.argtypes = [P, i32, i32, P, P, P, P]
+    L.tri_calib_finalize.restype = ctypes.c_int
     L.tri_last_cuda_error.argtypes = []
     L.tri_last_cuda_error.restype = ctypes.c_char_p
     _lib = L
@@ -310,3 +323,37 @@ class TriContext:
     def compress_launches(self, src: CacheView, dst: CacheView) -> int:
         a, b = src.c_view(), dst.c_view()
         return int(lib().tri_compress_launches(self._h, ctypes.byref(a), ctypes.byref(b)))
+
+
+class Calibrator:
+    """Streaming calibration statistics of one layer's query heads (Section 4.1): feed chunks of pre-RoPE
+    queries [T, n_heads, 128] (bf16 or fp32) with add(), read E[q_f], E|q_f| and R_f with result()."""
+
+    def __init__(self, n_heads: int, pair_layout: int = 0, device="cuda"):
+        self.n_heads, self.pair_layout, self.device = n_heads, pair_layout, torch.device(device)
+        self.state = torch.empty(lib().tri_calib_state_bytes(n_heads) // 8, dtype=torch.float64, device=self.device)
+        self._ws = None
+        self.reset()
+
+    def reset(self):
+        _check(lib().tri_calib_reset(_ptr(self.state), self.n_heads, _stream()), "tri_calib_reset")
+
+    def add(self, q: torch.Tensor):
+        assert q.dim() == 3 and q.shape[1] == self.n_heads and q.shape[2] == 128 and q.stride(2) == 1
+        assert q.dtype in (torch.bfloat16, torch.float32) and q.device == self.state.device
+        T = q.shape[0]
+        need = int(lib().tri_calib_workspace_bytes(self.n_heads, T))
+        if self._ws is None or self._ws.numel() * 8 < need:
+            self._ws = torch.empty((need + 7) // 8, dtype=torch.float64, device=self.device)
+        _check(lib().tri_calib_accumulate(_ptr(q), 0 if q.dtype == torch.bfloat16 else 1, T, self.n_heads, q.stride(0),
+                                          q.stride(1), self.pair_layout, _ptr(self.state), _ptr(self._ws),
+                                          self._ws.numel() * 8, _stream()), "tri_calib_accumulate")
+
+    def result(self):
+        """(q_center [n_heads, 128], q_mean_norm [n_heads, 64], mrl [n_heads, 64]) as fp32 device tensors."""
+        qc = torch.empty(self.n_heads, 128, dtype=torch.float32, device=self.device)
+        qn = torch.empty(self.n_heads, 64, dtype=torch.float32, device=self.device)
+        r = torch.empty(self.n_heads, 64, dtype=torch.float32, device=self.device)
+        _check(lib().tri_calib_finalize(_ptr(self.state), self.n_heads, self.pair_layout, _ptr(qc), _ptr(qn), _ptr(r),
+                                        _stream()), "tri_calib_finalize")
+        return qc, qn, r

@@ -8,6 +8,7 @@
 #include <new>
 #include <vector>
 
+#include "tri_calib.cuh"
 #include "tri_compact.cuh"
 #include "tri_score.cuh"
 #include "tri_score_tma.cuh"
@@ -611,4 +612,83 @@ extern "C" tri_status tri_score_static(tri_ctx *c, const tri_cache_view *src, in
     void *ws = nullptr;
     if ((r = score_scratch_address(dev, &ws)) != TRI_OK) return r;
     return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream);
+}
+
+// ----------------------------------------------------------------------------------------------
+// calibration statistics
+// ----------------------------------------------------------------------------------------------
+namespace {
+
+// Blocks per head and tokens per block: enough blocks to fill the GPU several times over, at least 256
+// tokens each, at most 1,024 blocks per head.
+void calib_shape(int32_t n_heads, int64_t T, int32_t *nblocks, int32_t *per_block)
+{
+    int64_t want = (148 * 16 + n_heads - 1) / n_heads;
+    int64_t most = (T + 255) / 256;
+    int64_t nb = want < most ? want : most;
+    if (nb > 1024) nb = 1024;
+    if (nb < 1) nb = 1;
+    int64_t per = (T + nb - 1) / nb;
+    *per_block = (int32_t)per;
+    *nblocks = (int32_t)((T + per - 1) / per);
+}
+
+}  // namespace
+
+extern "C" size_t tri_calib_state_bytes(int32_t n_heads)
+{
+    return n_heads > 0 ? ((size_t)n_heads * kCalibSums + 1) * sizeof(double) : 0;
+}
+
+extern "C" size_t tri_calib_workspace_bytes(int32_t n_heads, int64_t T)
+{
+    if (n_heads <= 0 || T <= 0) return 0;
+    int32_t nb, per;
+    calib_shape(n_heads, T, &nb, &per);
+    return (size_t)n_heads * nb * kCalibSums * sizeof(double);
+}
+
+extern "C" tri_status tri_calib_reset(void *state, int32_t n_heads, void *stream)
+{
+    if (!state || n_heads <= 0 || ((uintptr_t)state & 7)) return TRI_ERR_INVALID_ARG;
+    TRI_CUDA(cudaMemsetAsync(state, 0, tri_calib_state_bytes(n_heads), (cudaStream_t)stream));
+    return TRI_OK;
+}
+
+extern "C" tri_status tri_calib_accumulate(const void *q, int32_t q_kind, int64_t T, int32_t n_heads, int64_t stride_tok,
+                                           int64_t stride_head, int32_t pair_layout, void *state, void *ws,
+                                           size_t ws_bytes, void *stream)
+{
+    if (!q || !state || !ws || T <= 0 || n_heads <= 0 || n_heads > 65535) return TRI_ERR_INVALID_ARG;
+    if (q_kind < 0 || q_kind > 1 || pair_layout < 0 || pair_layout > 1) return TRI_ERR_INVALID_ARG;
+    if (stride_tok % 4 || stride_head % 4 || stride_head < kHeadDim || ((uintptr_t)q & (q_kind == 0 ? 7 : 15)))
+        return TRI_ERR_INVALID_ARG;
+    if (((uintptr_t)state & 7) || ((uintptr_t)ws & 7)) return TRI_ERR_INVALID_ARG;
+    if (ws_bytes < tri_calib_workspace_bytes(n_heads, T)) return TRI_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    CalibParams p;
+    p.q = q; p.T = T; p.stride_tok = stride_tok; p.stride_head = stride_head;
+    int32_t nb;
+    calib_shape(n_heads, T, &nb, &p.per_block);
+    p.partials = (double *)ws;
+    dim3 grid(nb, n_heads);
+    if (pair_layout == 0 && q_kind == 0) k_calib_partial<0, 0><<<grid, kCalibThreads, 0, st>>>(p);
+    else if (pair_layout == 0) k_calib_partial<0, 1><<<grid, kCalibThreads, 0, st>>>(p);
+    else if (q_kind == 0) k_calib_partial<1, 0><<<grid, kCalibThreads, 0, st>>>(p);
+    else k_calib_partial<1, 1><<<grid, kCalibThreads, 0, st>>>(p);
+    tri_status r = check_launch("k_calib_partial");
+    if (r != TRI_OK) return r;
+    k_calib_merge<<<n_heads, kCalibSums, 0, st>>>(p.partials, nb, T, (double *)state, n_heads);
+    return check_launch("k_calib_merge");
+}
+
+extern "C" tri_status tri_calib_finalize(const void *state, int32_t n_heads, int32_t pair_layout, float *q_center,
+                                         float *q_mean_norm, float *mrl, void *stream)
+{
+    if (!state || !q_center || !q_mean_norm || n_heads <= 0 || pair_layout < 0 || pair_layout > 1)
+        return TRI_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (pair_layout == 0) k_calib_finish<0><<<n_heads, kBands, 0, st>>>((const double *)state, n_heads, q_center, q_mean_norm, mrl);
+    else k_calib_finish<1><<<n_heads, kBands, 0, st>>>((const double *)state, n_heads, q_center, q_mean_norm, mrl);
+    return check_launch("k_calib_finish");
 }
