@@ -269,6 +269,39 @@ def test_compact_standalone_and_rerun_determinism():
     assert torch.equal(p2, a["pos_out"]) and lens.tolist() == [sp.budget]
 
 
+def test_round_replays_from_a_cuda_graph():
+    """tri_compress only enqueues kernels on the given stream (no allocation, no synchronisation), so a decode
+    loop can capture one round in a CUDA graph and replay it; the replay reads cur_pos from device memory."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="graph", n_layers=2, n_kv_heads=2, n_keys=6000, budget=500)
+    w = W.make_workload(sp, DEV)
+    direct = run_compress(w, sp.budget, want_scores=False)           # also the first call: one-time kernel set-up
+    ctx = direct["ctx"]
+    src = src_view(w)
+    U = 4
+    k2, v2 = torch.zeros_like(direct["k_out"]), torch.zeros_like(direct["v_out"])
+    p2 = torch.zeros_like(direct["pos_out"])
+    idx = torch.zeros(U, sp.budget, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(U, dtype=torch.int32, device=DEV)
+    ws = ctx.workspace(1, sp.n_keys, sp.budget)
+    cur = w.cur_pos.clone()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.compress(src, cur, sp.budget, tb.CacheView(k2, v2, positions=p2), ws, kept_idx=idx, kept_cnt=cnt)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(idx, direct["kept_idx"]) and torch.equal(cnt, direct["kept_cnt"])
+    assert torch.equal(k2.view(torch.int16), direct["k_out"].view(torch.int16)) and torch.equal(p2, direct["pos_out"])
+    # a later query position, written into the captured buffer, changes the scores of the replay
+    cur += 4096
+    w.cur_pos = cur.clone()
+    later = run_compress(w, sp.budget, ctx=ctx, want_scores=False)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(idx, later["kept_idx"]) and not torch.equal(idx, direct["kept_idx"])
+    assert torch.equal(v2.view(torch.int16), later["v_out"].view(torch.int16))
+
+
 def test_bad_page_id_sets_status_not_fault():
     """A page id outside the pool is reported through device_status; its rows are skipped."""
     sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name="badpage", n_layers=1, n_kv_heads=1, n_seqs=2, n_keys=400,
