@@ -9,7 +9,7 @@ import oracle
 from paper_2604_04921_b200 import binding as tb
 from paper_2604_04921_b200 import workloads as W
 
-from parity import (check_compacted, check_kept, check_scores, check_unit, make_ctx, oracle_unit, run_compress,
+from parity import (check_compacted, check_kept, check_scores, check_unit, make_ctx, oracle_unit, out_rows, run_compress,
                     src_view, unit_index)
 
 pytestmark = pytest.mark.gpu
@@ -102,6 +102,28 @@ def test_config4_shape_ragged_paged(in_place):
     assert res["new_seq_lens"].tolist() == [min(n, sp.budget) for n in lens]
     for u, ref in refs.items():
         check_unit(w, res, ref, *u, sp.budget)
+
+
+def test_token_major_page_layout():
+    """Pages stored [layer][page][slot][head][128] (head stride 128, slot stride H * 128): the view's strides
+    describe it, nothing else changes."""
+    sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name="tokmajor", n_layers=2, n_kv_heads=2, n_seqs=2, n_keys=1800,
+                                                  n_keys_min=400, budget=256)
+    w = W.make_workload(sp, DEV)
+    ref = run_compress(w, sp.budget)
+    # same pool, token-major in memory, exposed through a permuted (strided) view of the usual index order
+    w2 = W.Workload(sp, w.q_center, w.q_mean_norm, w.k.permute(0, 1, 3, 2, 4).contiguous().permute(0, 1, 3, 2, 4),
+                    w.v.permute(0, 1, 3, 2, 4).contiguous().permute(0, 1, 3, 2, 4), w.seq_lens, w.cur_pos, None, w.page_table)
+    assert w2.k.stride()[2:4] == (128, sp.n_kv_heads * 128)
+    res = run_compress(w2, sp.budget, in_place=True)
+    assert int(res["status"].item()) == 0
+    assert torch.equal(res["kept_idx"], ref["kept_idx"])
+    assert torch.equal(torch.nan_to_num(res["raw"]), torch.nan_to_num(ref["raw"]))      # unwritten entries stay NaN
+    for (l, s, h) in _all_units(w):
+        cnt = int(ref["kept_cnt"][unit_index(w, l, s, h)])
+        k_a, v_a, _ = out_rows(w, ref, l, s, h, cnt)
+        k_b, v_b, _ = out_rows(w2, res, l, s, h, cnt)
+        assert torch.equal(k_a.view(torch.int16), k_b.view(torch.int16)) and torch.equal(v_a.view(torch.int16), v_b.view(torch.int16))
 
 
 def test_in_place_contiguous_matches_out_of_place():
