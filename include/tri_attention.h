@@ -37,7 +37,10 @@ typedef enum {
     TRI_ERR_UNSUPPORTED = 2,   /* head_dim != 128, group_size > 16, page_size % 16 != 0, ...    */
     TRI_ERR_WORKSPACE = 3,     /* ws_bytes < tri_workspace_bytes(...)                           */
     TRI_ERR_CUDA = 4,          /* a CUDA runtime call failed; see tri_last_cuda_error()         */
-    TRI_ERR_DEVICE_CHECK = 5   /* (reported through *device_status, never returned)             */
+    TRI_ERR_DEVICE_CHECK = 5,  /* (reported through *device_status, never returned): a page id or
+                                  kept index outside its range; such rows are skipped              */
+    TRI_ERR_TIMEOUT = 6        /* (reported through *device_status): a bounded wait inside a kernel
+                                  ran out; the kernel returned normally, outputs are unspecified    */
 } tri_status;
 
 /* Model and method constants.  Host memory; copied by tri_create. */
@@ -230,6 +233,13 @@ tri_status tri_calib_accumulate(const void *q, int32_t q_kind, int64_t T, int32_
                                 void *stream);
 tri_status tri_calib_finalize(const void *state, int32_t n_heads, int32_t pair_layout, float *q_center,
                               float *q_mean_norm, float *mrl, void *stream);
+
+/*
+ * Self-test of the bounded wait the scoring kernel uses for its copy-engine barriers (the paper has no
+ * counterpart): one warp waits on a barrier that nothing ever completes, gives up after a short poll limit,
+ * writes TRI_ERR_TIMEOUT to *device_status (device int32) and returns normally.  The context stays usable.
+ */
+tri_status tri_selftest_bounded_wait(int32_t *device_status, void *stream);
 
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char *tri_last_cuda_error(void);

@@ -27,10 +27,10 @@ EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri
            "tri_compress", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_last_cuda_error",
            "tri_profile_begin", "tri_profile_read", "tri_profile_end",
            "tri_calib_state_bytes", "tri_calib_workspace_bytes", "tri_calib_reset", "tri_calib_accumulate",
-           "tri_calib_finalize"]
+           "tri_calib_finalize", "tri_selftest_bounded_wait"]
 
 STATUS = {0: "TRI_OK", 1: "TRI_ERR_INVALID_ARG", 2: "TRI_ERR_UNSUPPORTED", 3: "TRI_ERR_WORKSPACE",
-          4: "TRI_ERR_CUDA", 5: "TRI_ERR_DEVICE_CHECK"}
+          4: "TRI_ERR_CUDA", 5: "TRI_ERR_DEVICE_CHECK", 6: "TRI_ERR_TIMEOUT"}
 
 DEFAULT_OFFSETS = tuple(1 << j for j in range(17))   # D = {1, 2, 4, ..., 2^16} (Section 4.2)
 
@@ -123,6 +123,8 @@ def lib():
     L.tri_calib_accumulate.restype = ctypes.c_int
     L.tri_calib_finalize.argtypes = [P, i32, i32, P, P, P, P]
     L.tri_calib_finalize.restype = ctypes.c_int
+    L.tri_selftest_bounded_wait.argtypes = [P, P]
+    L.tri_selftest_bounded_wait.restype = ctypes.c_int
     L.tri_last_cuda_error.argtypes = []
     L.tri_last_cuda_error.restype = ctypes.c_char_p
     _lib = L

@@ -532,6 +532,13 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
     return TRI_OK;
 }
 
+extern "C" tri_status tri_selftest_bounded_wait(int32_t *device_status, void *stream)
+{
+    if (!device_status) return TRI_ERR_INVALID_ARG;
+    k_selftest_wait<<<1, 32, 0, (cudaStream_t)stream>>>(device_status);
+    return check_launch("k_selftest_wait");
+}
+
 // ----------------------------------------------------------------------------------------------
 // per-kernel timing of tri_compress (measurement aid)
 // ----------------------------------------------------------------------------------------------

@@ -26,7 +26,6 @@ constexpr int kStages = 2;
 constexpr int kTileBytes = kTileKeys * kHeadDim * 2;                       // 4096
 constexpr int kScoreDynSmem = kScoreWarps * kStages * kTileBytes;          // 65536: three blocks per SM
 constexpr uint32_t kWaitPolls = 1u << 22;                                  // bound on every mbarrier wait
-constexpr int TRI_STATUS_TIMEOUT = 6;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -50,10 +49,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
-// Waits for the phase with the given parity; gives up after kWaitPolls polls and returns false.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// Waits for the phase with the given parity; gives up after `polls` polls and returns false.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t polls = kWaitPolls)
 {
-    for (uint32_t i = 0; i < kWaitPolls; ++i)
+    for (uint32_t i = 0; i < polls; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -268,7 +267,7 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
     if (timed_out) {
         // a copy did not land within the bound: report it, give copies still in flight one more bounded
         // chance to land in this block's shared memory, and fall through to the block's normal exit
-        if (p.device_status) atomicExch(p.device_status, TRI_STATUS_TIMEOUT);
+        if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_TIMEOUT);
         for (int st = 0; st < kStages; ++st) (void)mbar_wait_bounded(my_bars + st * 8, 0);
     }
 
@@ -289,6 +288,20 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
         for (int w = 0; w < kScoreWarps; ++w) { a += red[w][tid][0]; b += red[w][tid][1]; }
         p.partials[((int64_t)u * p.nchunks + chunk) * G + tid] = make_double2(a, b);
     }
+}
+
+// One warp, one barrier that never completes: the wait must run out and report it (see tri_selftest_bounded_wait).
+__global__ void k_selftest_wait(int32_t *device_status)
+{
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncwarp();
+    const bool done = mbar_wait_bounded(b, 0, 1u << 12);
+    if (!done && threadIdx.x == 0) atomicExch(device_status, (int)TRI_ERR_TIMEOUT);
 }
 
 }  // namespace tri

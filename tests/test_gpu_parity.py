@@ -334,6 +334,18 @@ def test_bad_page_id_sets_status_not_fault():
     assert int(res["status"].item()) == 5
 
 
+def test_bounded_wait_runs_out_and_reports():
+    """The wait the scoring kernel uses for its copy barriers gives up after its poll limit: a barrier that
+    nothing completes yields status 6 (TRI_ERR_TIMEOUT), the kernel returns, and the device keeps working."""
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    assert tb.lib().tri_selftest_bounded_wait(status.data_ptr(), None) == 0
+    torch.cuda.synchronize()
+    assert int(status.item()) == 6
+    w = W.make_workload(W.SPECS["tiny"].scaled(name="afterwait", n_keys=500, budget=50), DEV)
+    res = run_compress(w, 50)
+    check_unit(w, res, oracle_unit(w, 0, 0, 0, 50), 0, 0, 0, 50)
+
+
 def test_host_errors_launch_nothing():
     w = W.make_workload(W.SPECS["tiny"].scaled(n_keys=256, budget=32), DEV)
     ctx = make_ctx(w)
