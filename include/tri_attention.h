@@ -152,9 +152,11 @@ tri_status tri_compress(tri_ctx *ctx, const tri_cache_view *src, int32_t S, cons
                         void *ws, size_t ws_bytes, void *stream);
 
 /*
- * The fused round for a cache that lives in HOST memory (contiguous views only): copies K, V
- * (and positions) of src to the device staging view, runs tri_compress, and copies the
- * compacted rows, positions and counts back, all on `stream`.
+ * The fused round for a cache that lives in HOST memory (contiguous views only): copies K of src to the
+ * device staging view, runs tri_compress, and copies the compacted rows, positions and counts back, all
+ * on `stream`.  V and positions are needed only for the kept rows: if their host arrays are pinned and
+ * mapped (cudaHostAlloc / cudaHostRegister), the gather reads those rows directly from host memory and no
+ * bulk copy of them is made; otherwise they are staged like K.
  *   src_host / dst_host  views whose k, v, positions, seq_lens pointers are (pinned) host memory
  *   src_dev  / dst_dev   device views of identical shape used as staging (caller-allocated)
  *   cur_pos_host         host [S] int64;  cur_pos_dev device [S] staging

@@ -509,16 +509,29 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
     const size_t kes = src_host->k_kind == 0 ? 2 : 4;
     const size_t src_elems = (size_t)L * src_host->stride_layer, dst_elems = (size_t)L * dst_host->stride_layer;
     const size_t U = (size_t)L * S * H;
+    // Keys are streamed in full by the scoring kernel, so they are copied.  Values and positions are only read
+    // for the kept rows: when the host arrays are device-accessible (pinned, mapped), the gather reads those
+    // rows straight from host memory and the bulk copies are skipped.
+    auto device_alias = [](const void *host_ptr) -> void * {
+        cudaPointerAttributes a;
+        if (!host_ptr || cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+    };
+    tri_cache_view sv = *src_dev;
     TRI_CUDA(cudaMemcpyAsync(src_dev->k, src_host->k, src_elems * kes, cudaMemcpyHostToDevice, st));
-    if (src_host->v && src_dev->v)
-        TRI_CUDA(cudaMemcpyAsync(src_dev->v, src_host->v, src_elems * 2, cudaMemcpyHostToDevice, st));
-    if (src_host->positions && src_dev->positions)
-        TRI_CUDA(cudaMemcpyAsync(src_dev->positions, src_host->positions, U * src_host->n_max * sizeof(int32_t),
-                                 cudaMemcpyHostToDevice, st));
+    if (src_host->v && src_dev->v) {
+        if (void *alias = device_alias(src_host->v)) sv.v = alias;
+        else TRI_CUDA(cudaMemcpyAsync(src_dev->v, src_host->v, src_elems * 2, cudaMemcpyHostToDevice, st));
+    }
+    if (src_host->positions && src_dev->positions) {
+        if (void *alias = device_alias(src_host->positions)) sv.positions = (int32_t *)alias;
+        else TRI_CUDA(cudaMemcpyAsync(src_dev->positions, src_host->positions, U * src_host->n_max * sizeof(int32_t),
+                                      cudaMemcpyHostToDevice, st));
+    }
     TRI_CUDA(cudaMemcpyAsync((void *)src_dev->seq_lens, src_host->seq_lens, S * sizeof(int32_t),
                              cudaMemcpyHostToDevice, st));
     TRI_CUDA(cudaMemcpyAsync(cur_pos_dev, cur_pos_host, S * sizeof(int64_t), cudaMemcpyHostToDevice, st));
-    tri_status r = tri_compress(c, src_dev, S, cur_pos_dev, budget, dst_dev, nullptr, kept_cnt_dev, nullptr, nullptr,
+    tri_status r = tri_compress(c, &sv, S, cur_pos_dev, budget, dst_dev, nullptr, kept_cnt_dev, nullptr, nullptr,
                                 ws, ws_bytes, stream);
     if (r != TRI_OK) return r;
     TRI_CUDA(cudaMemcpyAsync(dst_host->k, dst_dev->k, dst_elems * kes, cudaMemcpyDeviceToHost, st));

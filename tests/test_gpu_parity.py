@@ -291,6 +291,36 @@ def test_compact_standalone_and_rerun_determinism():
     assert torch.equal(p2, a["pos_out"]) and lens.tolist() == [sp.budget]
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_resident_cache_round(pinned):
+    """tri_compress_host: K/V/positions in host memory in, compacted rows in host memory out; with pinned
+    arrays V and positions are never copied in bulk (the gather reads the kept rows from host memory)."""
+    sp = W.SPECS["qwen3_8b_steady_b64"].scaled(name="hostpath", n_layers=2, n_kv_heads=2, n_seqs=3)
+    w = W.make_workload(sp, DEV)
+    ref = run_compress(w, sp.budget, want_scores=False)
+    L, S, H, B, N = 2, 3, 2, sp.budget, sp.n_keys
+    host = lambda t: (t.cpu().pin_memory() if pinned else t.cpu())
+    hk, hv, hpos = host(w.k), host(w.v), host(w.positions)
+    hlens, hcur = host(w.seq_lens), host(w.cur_pos)
+    hk2 = host(torch.zeros(L, S, H, B, 128, dtype=torch.bfloat16)); hv2 = host(torch.zeros_like(hk2))
+    hp2 = host(torch.zeros(L, S, H, B, dtype=torch.int32)); hcnt = host(torch.zeros(L * S * H, dtype=torch.int32))
+    dk = torch.empty_like(w.k); dv = torch.full_like(w.v, float("nan")); dpos = torch.full_like(w.positions, -7)
+    dlens, dcur = torch.empty_like(w.seq_lens), torch.empty_like(w.cur_pos)
+    k2 = torch.empty(L, S, H, B, 128, dtype=torch.bfloat16, device=DEV); v2 = torch.empty_like(k2)
+    p2 = torch.empty(L, S, H, B, dtype=torch.int32, device=DEV); cnt = torch.empty(L * S * H, dtype=torch.int32, device=DEV)
+    ctx = ref["ctx"]
+    ws = ctx.workspace(S, N, B)
+    ctx.compress_host(tb.CacheView(hk, hv, seq_lens=hlens, positions=hpos), tb.CacheView(dk, dv, seq_lens=dlens, positions=dpos),
+                      hcur, dcur, B, tb.CacheView(hk2, hv2, positions=hp2), tb.CacheView(k2, v2, positions=p2), hcnt, cnt, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(hcnt, ref["kept_cnt"].cpu())
+    assert torch.equal(hk2.view(torch.int16), ref["k_out"].cpu().view(torch.int16))
+    assert torch.equal(hv2.view(torch.int16), ref["v_out"].cpu().view(torch.int16))
+    assert torch.equal(hp2, ref["pos_out"].cpu())
+    if pinned:      # the staging copies of V and positions were never written
+        assert bool(torch.isnan(dv.float()).all()) and bool((dpos == -7).all())
+
+
 def test_round_replays_from_a_cuda_graph():
     """tri_compress only enqueues kernels on the given stream (no allocation, no synchronisation), so a decode
     loop can capture one round in a CUDA graph and replay it; the replay reads cur_pos from device memory."""
