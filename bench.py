@@ -450,7 +450,10 @@ def main():
         # K is copied in full; of V and the positions only the kept rows cross the link (read by the gather
         # straight from the pinned host arrays)
         kept_rows = sum(min(B, n) for n in lens) * L * H
-        h2d = hk.numel() * 2 + kept_rows * 256 + (0 if hpos is None else kept_rows * 4) + S * 12
+        if 2 * B <= n_max:
+            h2d = hk.numel() * 2 + kept_rows * 256 + (0 if hpos is None else kept_rows * 4) + S * 12
+        else:       # most rows are kept: V and positions are staged in bulk like K
+            h2d = (hk.numel() + hv.numel()) * 2 + (0 if hpos is None else hpos.numel() * 4) + S * 12
         d2h = (hk2.numel() + hv2.numel()) * 2 + hp2.numel() * 4 + U * 4
         line["e2e"] = {"value": whole_job_value(world, keys_per_step, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                        "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

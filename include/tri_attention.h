@@ -154,9 +154,13 @@ tri_status tri_compress(tri_ctx *ctx, const tri_cache_view *src, int32_t S, cons
 /*
  * The fused round for a cache that lives in HOST memory (contiguous views only): copies K of src to the
  * device staging view, runs tri_compress, and copies the compacted rows, positions and counts back, all
- * on `stream`.  V and positions are needed only for the kept rows: if their host arrays are pinned and
- * mapped (cudaHostAlloc / cudaHostRegister), the gather reads those rows directly from host memory and no
- * bulk copy of them is made; otherwise they are staged like K.
+ * on `stream`.  V and positions are needed only for the kept rows: if at most half of the rows can be kept
+ * (2 * budget <= n_max) and their host arrays are pinned and mapped (cudaHostAlloc / cudaHostRegister), the
+ * gather reads those rows directly from host memory and no bulk copy of them is made; otherwise they are
+ * staged like K.  The work is pipelined over up to 8 ranges of
+ * layers: a range's results travel back on a copy stream owned by the context while the next range is coming
+ * in; `stream` waits for that stream at the end, so work enqueued on it after the call sees the host outputs.
+ * One context must not run two tri_compress_host calls at once.
  *   src_host / dst_host  views whose k, v, positions, seq_lens pointers are (pinned) host memory
  *   src_dev  / dst_dev   device views of identical shape used as staging (caller-allocated)
  *   cur_pos_host         host [S] int64;  cur_pos_dev device [S] staging

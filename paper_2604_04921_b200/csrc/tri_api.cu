@@ -16,6 +16,7 @@
 
 using namespace tri;
 
+constexpr int kHostSlabs = 8;     // layer ranges tri_compress_host is pipelined over
 constexpr int kProfEvents = 6;   // boundaries of the 5 launches of tri_compress
 
 struct tri_ctx {
@@ -27,6 +28,11 @@ struct tri_ctx {
     float *mw_d;         // [L][H*G][64]   weight of |k_f| in the norm term
     bool profiling;      // tri_profile_begin .. tri_profile_end: time each kernel of tri_compress
     cudaEvent_t ev[kProfEvents];
+    // tri_compress_host: device-to-host copies of one layer range run on `back` while the caller's stream
+    // already brings in and compresses the next range
+    cudaStream_t back;
+    cudaEvent_t slab_done[kHostSlabs], back_done;
+    bool have_back;
 };
 
 // Records event i on the stream while profiling is on (between the launches of tri_compress).
@@ -73,6 +79,7 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
     c->desc.offsets = nullptr;
     c->omega_d = nullptr; c->dbar_d = nullptr; c->qc_d = nullptr; c->mw_d = nullptr;
     c->profiling = false;
+    c->have_back = false;
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaGetDevice"); }
 
@@ -110,6 +117,18 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
         if ((e = cudaMemcpy(c->dbar_d, dbar, sizeof dbar, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(c->qc_d, q_center, nq * kHeadDim * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(c->mw_d, mw.data(), nq * kBands * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaStreamCreateWithFlags(&c->back, cudaStreamNonBlocking)) != cudaSuccess) break;
+        int made = 0;
+        for (; made <= kHostSlabs; ++made)
+            if ((e = cudaEventCreateWithFlags(made < kHostSlabs ? &c->slab_done[made] : &c->back_done,
+                                              cudaEventDisableTiming)) != cudaSuccess)
+                break;
+        if (e != cudaSuccess) {
+            for (int i = 0; i < made; ++i) cudaEventDestroy(i < kHostSlabs ? c->slab_done[i] : c->back_done);
+            cudaStreamDestroy(c->back);
+            break;
+        }
+        c->have_back = true;
     } while (0);
     if (e != cudaSuccess) {
         st = cuda_fail(e, "tri_create");
@@ -124,6 +143,11 @@ extern "C" tri_status tri_destroy(tri_ctx *c)
 {
     if (!c) return TRI_OK;
     if (c->profiling) for (int i = 0; i < kProfEvents; ++i) cudaEventDestroy(c->ev[i]);
+    if (c->have_back) {
+        for (int i = 0; i < kHostSlabs; ++i) cudaEventDestroy(c->slab_done[i]);
+        cudaEventDestroy(c->back_done);
+        cudaStreamDestroy(c->back);
+    }
     cudaFree(c->omega_d);
     cudaFree(c->dbar_d);
     cudaFree(c->qc_d);
@@ -155,11 +179,14 @@ void pick_chunk(int32_t n_max, int32_t *chunk, int32_t *nchunks)
     *nchunks = (tiles + per - 1) / per;
 }
 
-Plan make_plan(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget)
+// A range of the context's layers; views handed down with it start at its first layer.
+struct Layers { int32_t first, count; };
+
+Plan make_plan(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget, int32_t n_layers = 0)
 {
     Plan p;
     const int G = c->desc.group_size;
-    p.U = c->desc.n_layers * S * c->desc.n_kv_heads;
+    p.U = (n_layers > 0 ? n_layers : c->desc.n_layers) * S * c->desc.n_kv_heads;
     pick_chunk(n_max, &p.chunk, &p.nchunks);
     size_t o = 0;
     p.off_E = o;      o += align256((size_t)S * kBands * sizeof(double2));
@@ -217,7 +244,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, CUtensorMap *out)
+tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, int32_t n_layers, CUtensorMap *out)
 {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
@@ -231,7 +258,7 @@ tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, 
     cuuint64_t dims[5], strides[4];
     dims[0] = kHeadDim;
     dims[2] = (cuuint64_t)c->desc.n_kv_heads;
-    dims[4] = (cuuint64_t)c->desc.n_layers;
+    dims[4] = (cuuint64_t)n_layers;
     if (v->paged) {
         dims[1] = (cuuint64_t)v->page_size;
         dims[3] = v->n_pages > 0 ? (cuuint64_t)v->n_pages : (cuuint64_t)0x7fffffff;
@@ -279,8 +306,11 @@ tri_status launch_score_tma(int NT, dim3 grid, cudaStream_t st, const CUtensorMa
 // fold -> raw scores -> z-score/max (3 launches); without the last one when `scores` is NULL: the fused round
 // leaves the normalisation to its selection kernel.
 tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, float *scores,
-                     float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st)
+                     float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st,
+                     Layers ly = Layers{0, 0})
 {
+    if (ly.count == 0) ly.count = c->desc.n_layers;
+    const size_t head0 = (size_t)ly.first * c->desc.n_kv_heads * c->desc.group_size;   // first query head of the range
     const int G = c->desc.group_size;
     double2 *E = (double2 *)(ws + pl.off_E);
     float *raw = raw_out ? raw_out : (float *)(ws + pl.off_raw);
@@ -296,13 +326,13 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     sp.src = to_view(src);
     sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G;
     sp.chunk = pl.chunk; sp.nchunks = pl.nchunks;
-    sp.E = E; sp.qc = c->qc_d; sp.mw = c->mw_d;
+    sp.E = E; sp.qc = c->qc_d + head0 * kHeadDim; sp.mw = c->mw_d + head0 * kBands;
     sp.raw = raw; sp.partials = part; sp.device_status = device_status;
     dim3 grid((unsigned)((size_t)pl.U * pl.nchunks));
     if (src->k_kind == 0) {
         int NT = G <= 4 ? 1 : (G <= 8 ? 2 : 4);
         CUtensorMap map;
-        if ((r = encode_key_map(c, src, S, &map)) != TRI_OK) return r;
+        if ((r = encode_key_map(c, src, S, ly.count, &map)) != TRI_OK) return r;
         r = c->desc.pair_layout == 0 ? launch_score_tma<0>(NT, grid, st, map, sp)
                                      : launch_score_tma<1>(NT, grid, st, map, sp);
         if (r != TRI_OK) return r;
@@ -456,6 +486,25 @@ extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const i
     return run_compact(c, src, kept_idx, kept_cnt, S, budget, dst, new_seq_lens, nullptr, U, (cudaStream_t)stream);
 }
 
+// The fused round over a range of layers; the views start at the range's first layer.
+static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                  int32_t budget, const tri_cache_view *dst, int32_t *kept_idx, int32_t *kept_cnt,
+                                  int32_t *new_seq_lens, int32_t *device_status, void *ws, size_t ws_bytes,
+                                  cudaStream_t st)
+{
+    tri_status r;
+    Plan pl = make_plan(c, S, src->n_max, budget, ly.count);
+    if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
+    char *w = (char *)ws;
+    int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
+    int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
+    if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, ly)) != TRI_OK) return r;
+    if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, &pl, w, st)) !=
+        TRI_OK)
+        return r;
+    return run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, pl.U, st);
+}
+
 extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                                    int32_t budget, const tri_cache_view *dst, int32_t *kept_idx,
                                    int32_t *kept_cnt, int32_t *new_seq_lens, int32_t *device_status,
@@ -469,17 +518,8 @@ extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_
     if (dst->n_max < budget && dst->n_max < src->n_max) return TRI_ERR_INVALID_ARG;
     if (src->k_kind != dst->k_kind) return TRI_ERR_INVALID_ARG;
     if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
-    Plan pl = make_plan(c, S, src->n_max, budget);
-    if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
-    char *w = (char *)ws;
-    int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
-    int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
-    if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st)) != TRI_OK) return r;
-    if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, &pl, w, st)) !=
-        TRI_OK)
-        return r;
-    return run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, pl.U, st);
+    return compress_layers(c, Layers{0, c->desc.n_layers}, src, S, cur_pos, budget, dst, kept_idx, kept_cnt, new_seq_lens,
+                           device_status, ws, ws_bytes, (cudaStream_t)stream);
 }
 
 extern "C" int32_t tri_compress_launches(const tri_ctx *c, const tri_cache_view *src, const tri_cache_view *dst)
@@ -504,11 +544,15 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
         src_host->n_max != src_dev->n_max || dst_host->n_max != dst_dev->n_max)
         return TRI_ERR_INVALID_ARG;
     if (!src_host->seq_lens || !src_dev->seq_lens || !src_host->k || !dst_host->k) return TRI_ERR_INVALID_ARG;
+    tri_status r;
+    if ((r = check_view(src_dev, true)) != TRI_OK) return r;
+    if ((r = check_view(dst_dev, false)) != TRI_OK) return r;
+    if ((r = check_common(c, S, src_dev->n_max, budget)) != TRI_OK) return r;
+    if (dst_dev->n_max < budget && dst_dev->n_max < src_dev->n_max) return TRI_ERR_INVALID_ARG;
+    if (src_dev->k_kind != dst_dev->k_kind || !ws || ((uintptr_t)ws & 255)) return TRI_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int L = c->desc.n_layers, H = c->desc.n_kv_heads;
     const size_t kes = src_host->k_kind == 0 ? 2 : 4;
-    const size_t src_elems = (size_t)L * src_host->stride_layer, dst_elems = (size_t)L * dst_host->stride_layer;
-    const size_t U = (size_t)L * S * H;
     // Keys are streamed in full by the scoring kernel, so they are copied.  Values and positions are only read
     // for the kept rows: when the host arrays are device-accessible (pinned, mapped), the gather reads those
     // rows straight from host memory and the bulk copies are skipped.
@@ -517,31 +561,68 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
         if (!host_ptr || cudaPointerGetAttributes(&a, host_ptr) != cudaSuccess) { cudaGetLastError(); return nullptr; }
         return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
     };
-    tri_cache_view sv = *src_dev;
-    TRI_CUDA(cudaMemcpyAsync(src_dev->k, src_host->k, src_elems * kes, cudaMemcpyHostToDevice, st));
-    if (src_host->v && src_dev->v) {
-        if (void *alias = device_alias(src_host->v)) sv.v = alias;
-        else TRI_CUDA(cudaMemcpyAsync(src_dev->v, src_host->v, src_elems * 2, cudaMemcpyHostToDevice, st));
-    }
-    if (src_host->positions && src_dev->positions) {
-        if (void *alias = device_alias(src_host->positions)) sv.positions = (int32_t *)alias;
-        else TRI_CUDA(cudaMemcpyAsync(src_dev->positions, src_host->positions, U * src_host->n_max * sizeof(int32_t),
-                                      cudaMemcpyHostToDevice, st));
-    }
+    // (in place only pays when most rows are dropped: row-sized reads across the link are slower than a bulk copy)
+    const bool sparse = 2 * (int64_t)budget <= src_dev->n_max;
+    void *v_alias = (sparse && src_host->v && src_dev->v) ? device_alias(src_host->v) : nullptr;
+    void *pos_alias = (sparse && src_host->positions && src_dev->positions) ? device_alias(src_host->positions) : nullptr;
     TRI_CUDA(cudaMemcpyAsync((void *)src_dev->seq_lens, src_host->seq_lens, S * sizeof(int32_t),
                              cudaMemcpyHostToDevice, st));
     TRI_CUDA(cudaMemcpyAsync(cur_pos_dev, cur_pos_host, S * sizeof(int64_t), cudaMemcpyHostToDevice, st));
-    tri_status r = tri_compress(c, &sv, S, cur_pos_dev, budget, dst_dev, nullptr, kept_cnt_dev, nullptr, nullptr,
-                                ws, ws_bytes, stream);
-    if (r != TRI_OK) return r;
-    TRI_CUDA(cudaMemcpyAsync(dst_host->k, dst_dev->k, dst_elems * kes, cudaMemcpyDeviceToHost, st));
-    if (dst_host->v && dst_dev->v)
-        TRI_CUDA(cudaMemcpyAsync(dst_host->v, dst_dev->v, dst_elems * 2, cudaMemcpyDeviceToHost, st));
-    if (dst_host->positions && dst_dev->positions)
-        TRI_CUDA(cudaMemcpyAsync(dst_host->positions, dst_dev->positions, U * dst_host->n_max * sizeof(int32_t),
-                                 cudaMemcpyDeviceToHost, st));
-    if (kept_cnt_host)
-        TRI_CUDA(cudaMemcpyAsync(kept_cnt_host, kept_cnt_dev, U * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+
+    // Layer ranges: range i is copied in and compressed on the caller's stream; its results go back to the host
+    // on the context's copy stream while range i + 1 is already coming in (the link is full duplex).
+    const int M = c->have_back ? (L < kHostSlabs ? L : kHostSlabs) : 1;
+    cudaStream_t back = M > 1 ? c->back : st;
+    const size_t upl = (size_t)S * H;                                  // units per layer
+    for (int i = 0; i < M; ++i) {
+        const int l0 = (int)((int64_t)L * i / M), nl = (int)((int64_t)L * (i + 1) / M) - l0;
+        const size_t so = (size_t)l0 * src_host->stride_layer, sn = (size_t)nl * src_host->stride_layer;
+        const size_t dof = (size_t)l0 * dst_host->stride_layer, dn = (size_t)nl * dst_host->stride_layer;
+        const size_t u0 = (size_t)l0 * upl, un = (size_t)nl * upl;
+        tri_cache_view sv = *src_dev, dv = *dst_dev;
+        sv.k = (char *)src_dev->k + so * kes;
+        TRI_CUDA(cudaMemcpyAsync(sv.k, (const char *)src_host->k + so * kes, sn * kes, cudaMemcpyHostToDevice, st));
+        if (src_host->v && src_dev->v) {
+            if (v_alias) {
+                sv.v = (char *)v_alias + so * 2;
+            } else {
+                sv.v = (char *)src_dev->v + so * 2;
+                TRI_CUDA(cudaMemcpyAsync(sv.v, (const char *)src_host->v + so * 2, sn * 2, cudaMemcpyHostToDevice, st));
+            }
+        }
+        if (src_host->positions && src_dev->positions) {
+            const size_t po = u0 * src_host->n_max, pn = un * src_host->n_max;
+            if (pos_alias) {
+                sv.positions = (int32_t *)pos_alias + po;
+            } else {
+                sv.positions = src_dev->positions + po;
+                TRI_CUDA(cudaMemcpyAsync(sv.positions, src_host->positions + po, pn * sizeof(int32_t),
+                                         cudaMemcpyHostToDevice, st));
+            }
+        }
+        dv.k = (char *)dst_dev->k + dof * kes;
+        if (dst_dev->v) dv.v = (char *)dst_dev->v + dof * 2;
+        if (dst_dev->positions) dv.positions = dst_dev->positions + u0 * dst_dev->n_max;
+        if ((r = compress_layers(c, Layers{l0, nl}, &sv, S, cur_pos_dev, budget, &dv, nullptr, kept_cnt_dev + u0, nullptr,
+                                 nullptr, ws, ws_bytes, st)) != TRI_OK)
+            return r;
+        if (M > 1) {
+            TRI_CUDA(cudaEventRecord(c->slab_done[i], st));
+            TRI_CUDA(cudaStreamWaitEvent(back, c->slab_done[i], 0));
+        }
+        TRI_CUDA(cudaMemcpyAsync((char *)dst_host->k + dof * kes, dv.k, dn * kes, cudaMemcpyDeviceToHost, back));
+        if (dst_host->v && dst_dev->v)
+            TRI_CUDA(cudaMemcpyAsync((char *)dst_host->v + dof * 2, dv.v, dn * 2, cudaMemcpyDeviceToHost, back));
+        if (dst_host->positions && dst_dev->positions)
+            TRI_CUDA(cudaMemcpyAsync(dst_host->positions + u0 * dst_host->n_max, dv.positions,
+                                     un * dst_host->n_max * sizeof(int32_t), cudaMemcpyDeviceToHost, back));
+        if (kept_cnt_host)
+            TRI_CUDA(cudaMemcpyAsync(kept_cnt_host + u0, kept_cnt_dev + u0, un * sizeof(int32_t), cudaMemcpyDeviceToHost, back));
+    }
+    if (M > 1) {
+        TRI_CUDA(cudaEventRecord(c->back_done, back));
+        TRI_CUDA(cudaStreamWaitEvent(st, c->back_done, 0));
+    }
     return TRI_OK;
 }
 
