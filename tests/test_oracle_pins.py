@@ -354,3 +354,25 @@ def test_calibration_matches_the_workload_generator_statistics():
         c, n, r = oracle.calibrate(q[:, hq].numpy())
         assert np.allclose(c, qc[0, hq].double().numpy(), atol=1e-6)
         assert np.allclose(n, qn[0, hq].double().numpy(), atol=1e-6)
+
+
+def test_oracle_reproduces_its_stored_config0_values():
+    """Regression guard: the oracle on the tiny configuration against the values its committed script stored
+    (tests/golden/make_config0_oracle.py, which calls only the oracle).  Floats to 1e-9 relative: libm's cos /
+    atan2 may differ in the last bits between machines; the kept set must be identical."""
+    import importlib.util
+    here = os.path.join(os.path.dirname(__file__), "golden")
+    spec = importlib.util.spec_from_file_location("make_config0_oracle", os.path.join(here, "make_config0_oracle.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    now = mod.render(*mod.compute()).splitlines()
+    stored = open(os.path.join(here, "config0_oracle.txt")).read().splitlines()
+    assert len(now) == len(stored)
+    for a, b in zip(now, stored):
+        ta, tb_ = a.split(), b.split()
+        if a.startswith("#") or ta[0].startswith("kept"):
+            assert a == b
+            continue
+        assert ta[0] == tb_[0]
+        for x, y in zip(ta[1:], tb_[1:]):
+            assert float(x) == pytest.approx(float(y), rel=1e-9, abs=1e-9)
