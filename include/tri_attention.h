@@ -67,7 +67,8 @@ typedef struct tri_ctx tri_ctx;
  * statistics of Section 4.1 and the offset-averaged phasors (1/|D|) sum_delta e^{i omega_f delta}.
  *   q_center     host [L][H*G][128] fp32  E[q_f]: pre-RoPE query centre, in the band layout above
  *   q_mean_norm  host [L][H*G][64]  fp32  E|q_f|
- * Allocates device memory (the only entry point besides tri_destroy that touches the allocator).
+ * Allocates device memory and creates the copy stream and events tri_compress_host uses (the only entry
+ * point besides tri_destroy and tri_profile_begin that allocates anything).
  */
 tri_status tri_create(const tri_model_desc *desc, const float *q_center, const float *q_mean_norm,
                       tri_ctx **out);
@@ -131,8 +132,10 @@ tri_status tri_select(tri_ctx *ctx, const float *scores, const int32_t *seq_lens
 
 /*
  * Eviction as an order-preserving gather (Section 4.3):  dst row j <- src row kept_idx[j] for K, V
- * and positions, j < kept_cnt[u].  dst may alias src (same k pointer and strides): the in-place
- * schedule then moves rows tile by tile in ascending order inside one thread block per unit.
+ * and positions, j < kept_cnt[u].  dst may alias src (same k pointer and strides): rows whose source lies
+ * inside the destination range [0, kept_cnt) are then moved tile by tile in ascending order by one thread
+ * block per unit (a tile is read completely before it is written), the rows behind them by a second,
+ * fully parallel launch; rows already in their slot are not touched.  kept_idx must be ascending.
  * dst->seq_lens is ignored; new_seq_lens (device [S], may be NULL) receives kept_cnt of the
  * sequence.  If dst->positions is given it receives the positions of the kept rows.
  */
@@ -144,7 +147,8 @@ tri_status tri_compact(tri_ctx *ctx, const tri_cache_view *src, const int32_t *k
  * The fused round: score, select, compact, in one call (a handful of launches, no host sync).
  *   kept_idx, kept_cnt   device outputs as in tri_select, or NULL to use workspace
  *   device_status        device int32[1] or NULL; set to TRI_ERR_DEVICE_CHECK if a kernel met a
- *                        page id outside [0, n_pages) -- such rows are skipped, never dereferenced
+ *                        page id outside [0, n_pages) -- such rows are skipped, never dereferenced --
+ *                        or to TRI_ERR_TIMEOUT if a bounded wait of the scoring kernel ran out
  */
 tri_status tri_compress(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                         int32_t budget, const tri_cache_view *dst, int32_t *kept_idx,
@@ -157,8 +161,7 @@ tri_status tri_compress(tri_ctx *ctx, const tri_cache_view *src, int32_t S, cons
  * on `stream`.  V and positions are needed only for the kept rows: if at most half of the rows can be kept
  * (2 * budget <= n_max) and their host arrays are pinned and mapped (cudaHostAlloc / cudaHostRegister), the
  * gather reads those rows directly from host memory and no bulk copy of them is made; otherwise they are
- * staged like K.  The work is pipelined over up to 8 ranges of
- * layers: a range's results travel back on a copy stream owned by the context while the next range is coming
+ * staged like K.  The work is pipelined over up to 8 ranges of layers: a range's results travel back on a copy stream owned by the context while the next range is coming
  * in; `stream` waits for that stream at the end, so work enqueued on it after the call sees the host outputs.
  * One context must not run two tri_compress_host calls at once.
  *   src_host / dst_host  views whose k, v, positions, seq_lens pointers are (pinned) host memory
