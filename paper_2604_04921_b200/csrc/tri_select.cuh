@@ -11,7 +11,9 @@
 //      equal scores, say) the same radix sweeps the unit's keys instead.
 //   3. emit in index order: the unit is cut into spans of at most 32 keys per thread; inside a span warp w
 //      owns a contiguous run of keys, 32 at a time, so warp ballots are already in index order and one
-//      block-wide scan of the warp totals per span places every kept slot.
+//      block-wide scan of the warp totals per span places every kept slot.  When few keys are kept the
+//      warp transposes its kept-bit matrix with ballots so that each lane places the kept keys of one row
+//      of 32 (work follows the number kept, not the number scanned).
 //
 // FUSED = true folds the GQA normalise-then-aggregate step into sweep 1: the final score is computed from
 // the raw per-head scores and the unit's (mu_g, 1/sigma_g), parked in the score buffer for the later
@@ -208,36 +210,73 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
 
     // ---- emit kept slots in ascending order; among keys equal to T the lowest slots win ----
     // J keys per thread and span (at most 32, fewer for short units so that no sweep runs empty)
-    const uint32_t lt = (1u << lane) - 1u;
     const int J = min(32, (n + kSelThreads - 1) / kSelThreads);
+    const bool dense = 2 * p.budget > n;        // more than half of the keys are kept
     uint32_t base = 0, need_rem = need;
 #pragma unroll 1
     for (int span = 0; span < n; span += kSelThreads * J) {
         const int ibase = span + warp * (32 * J) + lane;
-        uint32_t m_gt = 0, m_eq = 0, w_gt = 0, w_eq = 0;     // bit j: key ibase + 32 j is above / equal to T
-#pragma unroll 4
-        for (int j = 0; j < J; ++j) {
+        uint32_t m_gt = 0, m_eq = 0;                          // bit j: key ibase + 32 j is above / equal to T
+#pragma unroll 8
+        for (int j = 0; j < J; ++j) {                         // loads only: many in flight
             const int i = ibase + 32 * j;
             const uint32_t k = i < n ? float_key(sc[i]) : 0u;  // 0 is below every real key
-            const bool g = k > T, e = k == T;
-            m_gt |= (uint32_t)g << j;
-            m_eq |= (uint32_t)e << j;
-            w_gt += __popc(__ballot_sync(0xffffffffu, g));
-            w_eq += __popc(__ballot_sync(0xffffffffu, e));
+            m_gt |= (uint32_t)(k > T) << j;
+            m_eq |= (uint32_t)(k == T) << j;
+        }
+        uint32_t w_gt = __popc(m_gt), w_eq = __popc(m_eq);     // this warp's totals
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            w_gt += __shfl_xor_sync(0xffffffffu, w_gt, d);
+            w_eq += __shfl_xor_sync(0xffffffffu, w_eq, d);
         }
         // a span holds at most 32,768 keys, so the two 16-bit halves never carry into each other
         uint32_t total;
         uint32_t pre = block_excl_scan<THREADS>(lane == 0 ? (w_gt | (w_eq << 16)) : 0u, warp_sums, &total);
         pre = __shfl_sync(0xffffffffu, pre, 0);
-        uint32_t gt_before = pre & 0xffffu, eq_before = pre >> 16;
-        for (int j = 0; j < J; ++j) {
-            const bool g = m_gt >> j & 1u, e = m_eq >> j & 1u;
-            const uint32_t bg = __ballot_sync(0xffffffffu, g), be = __ballot_sync(0xffffffffu, e);
-            const uint32_t gb = gt_before + __popc(bg & lt), eb = eq_before + __popc(be & lt);
-            if (g) out[base + gb + min(eb, need_rem)] = ibase + 32 * j;
-            else if (e && eb < need_rem) out[base + gb + eb] = ibase + 32 * j;
-            gt_before += __popc(bg);
-            eq_before += __popc(be);
+        const uint32_t gt_before = pre & 0xffffu, eq_before = pre >> 16;
+        if (dense) {
+            // most keys are kept: walk the J slots in order, every lane places its own key
+            const uint32_t lt = (1u << lane) - 1u;
+            uint32_t gb0 = gt_before, eb0 = eq_before;
+            for (int j = 0; j < J; ++j) {
+                const bool g = m_gt >> j & 1u, e = m_eq >> j & 1u;
+                const uint32_t bg = __ballot_sync(0xffffffffu, g), be = __ballot_sync(0xffffffffu, e);
+                const uint32_t gb = gb0 + __popc(bg & lt), eb = eb0 + __popc(be & lt);
+                if (g) out[base + gb + min(eb, need_rem)] = ibase + 32 * j;
+                else if (e && eb < need_rem) out[base + gb + eb] = ibase + 32 * j;
+                gb0 += __popc(bg);
+                eb0 += __popc(be);
+            }
+        } else {
+            // Transpose the warp's 32 x J bit matrices: lane j ends up with row j (the keys ibase_w + 32 j + 0..31, one
+            // bit per key), so that each lane places the kept keys of one row and work follows the number kept.
+            uint32_t row_gt = 0, row_eq = 0;
+#pragma unroll 8
+            for (int j = 0; j < J; ++j) {
+                const uint32_t bg = __ballot_sync(0xffffffffu, m_gt >> j & 1u), be = __ballot_sync(0xffffffffu, m_eq >> j & 1u);
+                if (lane == j) { row_gt = bg; row_eq = be; }
+            }
+            const uint32_t cg = __popc(row_gt), ce = __popc(row_eq);
+            uint32_t sg = cg, se = ce;                              // inclusive scans over the rows (lanes)
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t yg = __shfl_up_sync(0xffffffffu, sg, d), ye = __shfl_up_sync(0xffffffffu, se, d);
+                if (lane >= d) { sg += yg; se += ye; }
+            }
+            const uint32_t g0 = gt_before + sg - cg, e0 = eq_before + se - ce;   // kept-above / equal keys before this row
+            const int rbase = span + warp * (32 * J) + 32 * lane;                 // slot of the row's first key
+            for (uint32_t r = row_gt; r; r &= r - 1) {
+                const int l = __ffs(r) - 1;
+                const uint32_t low = (1u << l) - 1u;
+                out[base + g0 + __popc(row_gt & low) + min(e0 + __popc(row_eq & low), need_rem)] = rbase + l;
+            }
+            for (uint32_t r = row_eq; r; r &= r - 1) {
+                const int l = __ffs(r) - 1;
+                const uint32_t low = (1u << l) - 1u;
+                const uint32_t eb = e0 + __popc(row_eq & low);
+                if (eb < need_rem) out[base + g0 + __popc(row_gt & low) + eb] = rbase + l;
+            }
         }
         const uint32_t te = min(total >> 16, need_rem);
         base += (total & 0xffffu) + te;
