@@ -8,6 +8,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "tri_calib.cuh"
 #include "tri_compact.cuh"
 #include "tri_score.cuh"
@@ -40,6 +42,12 @@ static void mark(tri_ctx *c, int i, cudaStream_t st)
 {
     if (c->profiling) cudaEventRecord(c->ev[i], st);
 }
+
+// Named range on the calling host thread for timeline tools (a no-op when no tool is attached).
+struct NvtxRange {
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 static thread_local char g_err[256] = "";
 
@@ -493,15 +501,23 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
                                   cudaStream_t st)
 {
     tri_status r;
+    NvtxRange whole("tri_compress");
     Plan pl = make_plan(c, S, src->n_max, budget, ly.count);
     if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
     char *w = (char *)ws;
     int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
     int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
-    if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, ly)) != TRI_OK) return r;
-    if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, &pl, w, st)) !=
-        TRI_OK)
-        return r;
+    {
+        NvtxRange part("tri_compress: fold + score");
+        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, ly)) != TRI_OK) return r;
+    }
+    {
+        NvtxRange part("tri_compress: normalise + select");
+        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, &pl, w,
+                            st)) != TRI_OK)
+            return r;
+    }
+    NvtxRange part("tri_compress: compact");
     return run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, pl.U, st);
 }
 
@@ -545,6 +561,7 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
         return TRI_ERR_INVALID_ARG;
     if (!src_host->seq_lens || !src_dev->seq_lens || !src_host->k || !dst_host->k) return TRI_ERR_INVALID_ARG;
     tri_status r;
+    NvtxRange whole("tri_compress_host");
     if ((r = check_view(src_dev, true)) != TRI_OK) return r;
     if ((r = check_view(dst_dev, false)) != TRI_OK) return r;
     if ((r = check_common(c, S, src_dev->n_max, budget)) != TRI_OK) return r;
