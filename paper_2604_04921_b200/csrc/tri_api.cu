@@ -216,6 +216,10 @@ View to_view(const tri_cache_view *v)
     w.stride_head = v->stride_head; w.stride_tok = v->stride_tok;
     w.page_table = v->page_table; w.max_pages_per_seq = v->max_pages_per_seq;
     w.page_size = v->page_size; w.n_pages = v->n_pages;
+    w.page_shift = -1;
+    if (v->page_size > 0 && (v->page_size & (v->page_size - 1)) == 0)
+        for (int sh = 0; sh < 31; ++sh)
+            if ((1 << sh) == v->page_size) w.page_shift = sh;
     w.stride_page = v->stride_page; w.stride_slot = v->stride_slot;
     w.seq_lens = v->seq_lens; w.positions = v->positions; w.n_max = v->n_max;
     return w;

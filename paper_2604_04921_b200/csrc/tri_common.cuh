@@ -22,6 +22,7 @@ struct View {
     int64_t stride_layer, stride_seq, stride_head, stride_tok;
     const int32_t *page_table;
     int32_t max_pages_per_seq, page_size, n_pages;
+    int32_t page_shift;        // log2(page_size) when it is a power of two, else -1 (host-derived)
     int64_t stride_page, stride_slot;
     const int32_t *seq_lens;
     int32_t *positions;
@@ -34,7 +35,7 @@ __device__ __forceinline__ int64_t row_offset(const View &w, int l, int s, int h
     if (!w.paged)
         return (int64_t)l * w.stride_layer + (int64_t)s * w.stride_seq + (int64_t)h * w.stride_head +
                (int64_t)n * w.stride_tok;
-    int pg = n / w.page_size;
+    const int pg = w.page_shift >= 0 ? n >> w.page_shift : n / w.page_size;
     int page = __ldg(w.page_table + (int64_t)s * w.max_pages_per_seq + pg);
     if (w.n_pages > 0 && (page < 0 || page >= w.n_pages)) return -1;
     return (int64_t)l * w.stride_layer + (int64_t)page * w.stride_page + (int64_t)h * w.stride_head +

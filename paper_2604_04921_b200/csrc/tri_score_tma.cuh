@@ -126,7 +126,7 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
         const int row = key_begin + (warp + kScoreWarps * it) * kTileKeys;
         int c1 = row, c3 = s;
         if (p.src.paged) {
-            const int pg = row / p.src.page_size;
+            const int pg = p.src.page_shift >= 0 ? row >> p.src.page_shift : row / p.src.page_size;
             int page = __ldg(p.src.page_table + (int64_t)s * p.src.max_pages_per_seq + pg);
             if (p.src.n_pages > 0 && (page < 0 || page >= p.src.n_pages)) {
                 if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
