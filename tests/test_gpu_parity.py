@@ -217,6 +217,34 @@ def test_degenerate_sizes():
     assert torch.all(res["k_out"][0, 1] == 0)
 
 
+def test_random_shapes_against_oracle():
+    """Twenty seeded random shapes (layers, heads, group size, batch, lengths, budget; contiguous, steady-state
+    positions or paged; in place or not) -- every unit against the oracle."""
+    import random
+    rnd = random.Random(20260404)
+    for case in range(20):
+        kind = rnd.choice(["oneshot", "steady", "ragged_paged"])
+        L, H, G, S = rnd.randint(1, 2), rnd.randint(1, 3), rnd.choice([1, 2, 3, 4, 6, 8]), rnd.randint(1, 3)
+        N = rnd.choice([17, 100, 333, 1024, 1999, 3100])
+        B = max(1, min(N + 50, int(N * rnd.choice([0.05, 0.3, 0.9, 1.2]))))
+        base = {"oneshot": "qwen3_8b_oneshot_32k", "steady": "qwen3_8b_steady_b64", "ragged_paged": "qwen3_32b_ragged_paged"}[kind]
+        extra = {}
+        if kind == "steady":
+            N = max(N, 200)
+            extra = dict(n_new=min(128, N // 2), pos_lo=N, pos_hi=N + 5000)
+        if kind == "ragged_paged":
+            extra = dict(n_keys_min=max(1, N // 4))
+        sp = W.SPECS[base].scaled(name=f"rand{case}", n_layers=L, n_kv_heads=H, group_size=G, n_seqs=S, n_keys=N,
+                                  budget=B, **extra)
+        w = W.make_workload(sp, DEV)
+        in_place = kind != "oneshot" and rnd.random() < 0.5
+        refs = {u: oracle_unit(w, *u, B) for u in _all_units(w)}       # before any in-place write
+        res = run_compress(w, B, in_place=in_place)
+        assert int(res["status"].item()) == 0, (case, kind)
+        for u, ref in refs.items():
+            check_unit(w, res, ref, *u, B)
+
+
 def test_constant_head_contributes_zero():
     """A query head with zero centre and E|q_f| = 0 scores every key 0: sigma = 0, z = 0 for that head."""
     sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="const", n_layers=1, n_kv_heads=1, group_size=2, n_keys=900,
