@@ -36,11 +36,11 @@ NOMINAL_HBM_GBS = 8000.0
 
 
 # DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum on
-# 1,048,576 keys: 268.562688 MB + 15.030272 MB), valid only for the kernel source it was taken on.
-SCORE_TRAFFIC = {"bytes_per_key": (268562688 + 15030272) / 1048576,
+# 1,048,576 keys: 268.562688 MB + 15.422976 MB), valid only for the kernel source it was taken on.
+SCORE_TRAFFIC = {"bytes_per_key": (268562688 + 15422976) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
-                 "sha256": "4efb7ee835935b415f830b6806653bfb423a1bdda6a7f99d62bb19dda332cf05"}
+                 "sha256": "f7ee43878b5afb27fa723650e902308bf21f043b7cf31fdc68ffa26346e2cd87"}
 
 
 def score_traffic_per_launch(keys):
