@@ -40,7 +40,7 @@ NOMINAL_HBM_GBS = 8000.0
 SCORE_TRAFFIC = {"bytes_per_key": (268562688 + 15422976) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
-                 "sha256": "f7ee43878b5afb27fa723650e902308bf21f043b7cf31fdc68ffa26346e2cd87"}
+                 "sha256": "f732a90f8607130c89fe05b59d9091a3e58e1ac37d4ac1008fe7c2a7f99acfa7"}
 
 
 def score_traffic_per_launch(keys):

@@ -145,6 +145,9 @@ tri_status tri_compact(tri_ctx *ctx, const tri_cache_view *src, const int32_t *k
 
 /*
  * The fused round: score, select, compact, in one call (a handful of launches, no host sync).
+ * Sequences with seq_lens[s] <= budget are kept whole (Section 4.3: pruning happens "if the cache exceeds
+ * budget B"): their keys are neither scored nor read, so a batch in which only some sequences are due costs
+ * only those.
  *   kept_idx, kept_cnt   device outputs as in tri_select, or NULL to use workspace
  *   device_status        device int32[1] or NULL; set to TRI_ERR_DEVICE_CHECK if a kernel met a
  *                        page id outside [0, n_pages) -- such rows are skipped, never dereferenced --

@@ -319,7 +319,7 @@ tri_status launch_score_tma(int NT, dim3 grid, cudaStream_t st, const CUtensorMa
 // leaves the normalisation to its selection kernel.
 tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, float *scores,
                      float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st,
-                     Layers ly = Layers{0, 0})
+                     Layers ly = Layers{0, 0}, int32_t skip_upto = 0)
 {
     if (ly.count == 0) ly.count = c->desc.n_layers;
     const size_t head0 = (size_t)ly.first * c->desc.n_kv_heads * c->desc.group_size;   // first query head of the range
@@ -336,7 +336,7 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
 
     ScoreParams sp;
     sp.src = to_view(src);
-    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G;
+    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G; sp.skip_upto = skip_upto;
     sp.chunk = pl.chunk; sp.nchunks = pl.nchunks;
     sp.E = E; sp.qc = c->qc_d + head0 * kHeadDim; sp.mw = c->mw_d + head0 * kBands;
     sp.raw = raw; sp.partials = part; sp.device_status = device_status;
@@ -513,7 +513,8 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
     int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
     {
         NvtxRange part("tri_compress: fold + score");
-        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, ly)) != TRI_OK) return r;
+        // sequences that do not exceed the budget are kept whole: their keys are not even read
+        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, ly, budget)) != TRI_OK) return r;
     }
     {
         NvtxRange part("tri_compress: normalise + select");

@@ -91,6 +91,7 @@ __device__ __forceinline__ uint32_t bf16_hi_bits(float w)   // bf16(w), round to
 struct ScoreParams {
     View src;
     int32_t S, H, G;
+    int32_t skip_upto;    // units of at most this many keys are not scored (the fused round keeps them whole); 0 = score all
     int32_t chunk;        // keys per block (multiple of 16)
     int32_t nchunks;      // blocks per unit
     const double2 *E;     // [S][64]  e^{i omega_f p_q} Dbar_f
@@ -117,7 +118,7 @@ k_score_f32_pre(const ScoreParams p, const double *__restrict__ omega, const dou
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int n = min(__ldg(p.src.seq_lens + s), p.src.n_max);
     const int key_begin = chunk * p.chunk;
-    if (key_begin >= n) return;
+    if (key_begin >= n || n <= p.skip_upto) return;
     const int key_end = min(key_begin + p.chunk, n);
     const int G = p.G;
     const int64_t pq = cur_pos[s];

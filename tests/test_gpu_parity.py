@@ -245,6 +245,26 @@ def test_random_shapes_against_oracle():
             check_unit(w, res, ref, *u, B)
 
 
+def test_only_overflowing_sequences_are_touched():
+    """A batch in which one sequence exceeds the budget and two do not: the short ones are kept whole, in order,
+    and the round gives the same kept rows for the long one as a batch holding it alone."""
+    base = W.SPECS["qwen3_8b_oneshot_32k"]
+    sp = base.scaled(name="due", n_layers=1, n_kv_heads=2, n_seqs=3, n_keys=900, budget=256)
+    w = W.make_workload(sp, DEV)
+    w.seq_lens = torch.tensor([200, 900, 256], dtype=torch.int32, device=DEV)
+    w.cur_pos = torch.tensor([200, 900, 256], dtype=torch.int64, device=DEV)
+    res = run_compress(w, 256, want_scores=False)
+    assert res["kept_cnt"].tolist() == [200, 200, 256, 256, 256, 256]
+    assert res["new_seq_lens"].tolist() == [200, 256, 256]
+    for s_, n_ in ((0, 200), (2, 256)):
+        for h in range(2):
+            u = unit_index(w, 0, s_, h)
+            assert res["kept_idx"][u, :n_].tolist() == list(range(n_))
+            assert torch.equal(res["k_out"][0, s_, h, :n_].view(torch.int16), w.k[0, s_, h, :n_].view(torch.int16))
+    for h in range(2):
+        check_unit(w, res, oracle_unit(w, 0, 1, h, 256), 0, 1, h, 256)
+
+
 def test_constant_head_contributes_zero():
     """A query head with zero centre and E|q_f| = 0 scores every key 0: sigma = 0, z = 0 for that head."""
     sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="const", n_layers=1, n_kv_heads=1, group_size=2, n_keys=900,
