@@ -245,6 +245,54 @@ def test_random_shapes_against_oracle():
             check_unit(w, res, ref, *u, B)
 
 
+def test_decode_windows_in_place_over_several_rounds():
+    """The deployed loop (Section 4.3): every 128 decoded tokens the cache, budget + 128 rows, is compressed in
+    place back to the budget; survivors keep their original positions.  Four rounds on the device against the
+    oracle applied to the same evolving cache on the host."""
+    B, beta, rounds = 384, 128, 4
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="loop", n_layers=1, n_kv_heads=2, n_keys=B + beta * rounds, budget=B)
+    full = W.make_workload(sp, DEV)                     # the whole decode: slot i = position i
+    L, S, H, G, cap = 1, 1, 2, sp.group_size, B + beta
+    k = torch.zeros(L, S, H, cap, 128, dtype=torch.bfloat16, device=DEV); v = torch.zeros_like(k)
+    pos = torch.zeros(L, S, H, cap, dtype=torch.int32, device=DEV)
+    k[..., :B, :], v[..., :B, :] = full.k[..., :B, :], full.v[..., :B, :]
+    pos[..., :B] = torch.arange(B, dtype=torch.int32, device=DEV)
+    lens = torch.tensor([B], dtype=torch.int32, device=DEV)
+    ctx = make_ctx(full)
+    ws = ctx.workspace(S, cap, B)
+    view = tb.CacheView(k, v, seq_lens=lens, positions=pos)
+    host = [dict(k=full.k[0, 0, h, :B].cpu(), v=full.v[0, 0, h, :B].cpu(), pos=torch.arange(B)) for h in range(H)]
+    for r in range(rounds):
+        t0 = B + beta * r                               # the window's tokens: positions t0 .. t0 + beta - 1
+        k[..., B:, :], v[..., B:, :] = full.k[..., t0:t0 + beta, :], full.v[..., t0:t0 + beta, :]
+        pos[..., B:] = torch.arange(t0, t0 + beta, dtype=torch.int32, device=DEV)
+        lens.fill_(cap)
+        cur = torch.tensor([t0 + beta], dtype=torch.int64, device=DEV)
+        ctx.compress(view, cur, B, view, ws, new_seq_lens=lens)
+        torch.cuda.synchronize()
+        assert lens.tolist() == [B]
+        for h in range(H):
+            st = host[h]
+            kk = torch.cat([st["k"], full.k[0, 0, h, t0:t0 + beta].cpu()])
+            vv = torch.cat([st["v"], full.v[0, 0, h, t0:t0 + beta].cpu()])
+            pp = torch.cat([st["pos"], torch.arange(t0, t0 + beta)])
+            _, s_o, idx_o = oracle.unit_bf16(W.bf16_bits(kk), pp.numpy(), t0 + beta, full.q_center[0, h * G:(h + 1) * G].double().numpy(),
+                                             full.q_mean_norm[0, h * G:(h + 1) * G].double().numpy(), B, theta=sp.theta)
+            got_pos = pos[0, 0, h, :B].cpu().long()
+            want_pos = pp[torch.from_numpy(idx_o.astype(np.int64))]
+            if not torch.equal(got_pos, want_pos):     # only keys in the tie band may differ
+                diff = np.setxor1d(got_pos.numpy(), want_pos.numpy())
+                s_b = np.sort(s_o)[::-1][B - 1]
+                where = np.isin(pp.numpy(), diff)
+                assert np.all(np.abs(s_o[where] - s_b) <= 1e-3 * max(1.0, abs(s_b)))
+                pytest.skip("a tie-band swap made the device and host caches diverge; later rounds are not comparable")
+            sel = torch.from_numpy(idx_o.astype(np.int64))
+            assert torch.equal(k[0, 0, h, :B].cpu().view(torch.int16), kk[sel].view(torch.int16))
+            assert torch.equal(v[0, 0, h, :B].cpu().view(torch.int16), vv[sel].view(torch.int16))
+            assert torch.all(got_pos[1:] > got_pos[:-1])
+            host[h] = dict(k=kk[sel], v=vv[sel], pos=want_pos)
+
+
 def test_only_overflowing_sequences_are_touched():
     """A batch in which one sequence exceeds the budget and two do not: the short ones are kept whole, in order,
     and the round gives the same kept rows for the long one as a batch holding it alone."""
