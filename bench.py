@@ -36,8 +36,8 @@ NOMINAL_HBM_GBS = 8000.0
 
 
 # DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum on
-# 1,048,576 keys: 268.562688 MB + 15.422976 MB), valid only for the kernel source it was taken on.
-SCORE_TRAFFIC = {"bytes_per_key": (268562688 + 15422976) / 1048576,
+# 1,048,576 keys: 268.564992 MB + 13.988352 MB), valid only for the kernel source it was taken on.
+SCORE_TRAFFIC = {"bytes_per_key": (268564992 + 13988352) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
                  "sha256": "f732a90f8607130c89fe05b59d9091a3e58e1ac37d4ac1008fe7c2a7f99acfa7"}
