@@ -145,10 +145,13 @@ tri_status tri_compact(tri_ctx *ctx, const tri_cache_view *src, const int32_t *k
 
 /*
  * The fused round: score, select, compact, in one call (a handful of launches, no host sync).
- * Sequences with seq_lens[s] <= budget are kept whole (Section 4.3: pruning happens "if the cache exceeds
- * budget B"): their keys are neither scored nor read, so a batch in which only some sequences are due costs
+ * Sequences with seq_lens[s] <= budget are kept whole (Section 4.3 prunes only a cache that has outgrown its
+ * budget): their keys are neither scored nor read, so a batch in which only some sequences are due costs
  * only those.
  *   kept_idx, kept_cnt   device outputs as in tri_select, or NULL to use workspace
+ *   new_seq_lens         device [S] or NULL: receives min(budget, seq_lens[s]).  It MAY be the same array as
+ *                        src->seq_lens (a decode loop that updates its lengths in place): the lengths are
+ *                        stored by the last launch of the round only, after every kernel that reads them.
  *   device_status        device int32[1] or NULL; set to TRI_ERR_DEVICE_CHECK if a kernel met a
  *                        page id outside [0, n_pages) -- such rows are skipped, never dereferenced --
  *                        or to TRI_ERR_TIMEOUT if a bounded wait of the scoring kernel ran out
@@ -223,7 +226,7 @@ tri_status tri_profile_read(tri_ctx *ctx, float *ms);
 tri_status tri_profile_end(tri_ctx *ctx);
 
 /*
- * Calibration statistics (Section 4.1: "computed from calibration data"; Section 3.3; Appendix B.5).
+ * Calibration statistics (Section 4.1 takes E[q_f] and E|q_f| from a calibration set; Section 3.3; Appendix B.5).
  * For one layer's query heads, from pre-RoPE query vectors of calibration tokens:
  *   E[q_f]   complex mean per band              -> q_center    [n_heads][128] fp32, in the input's component layout
  *   E|q_f|   mean band magnitude                -> q_mean_norm [n_heads][64]  fp32

@@ -64,6 +64,10 @@ static tri_status cuda_fail(cudaError_t e, const char *what)
 
 extern "C" const char *tri_last_cuda_error(void) { return g_err; }
 
+namespace {
+cudaError_t prepare_device();   // per-device kernel attributes, defined with the launch helpers below
+}
+
 // ----------------------------------------------------------------------------------------------
 // context
 // ----------------------------------------------------------------------------------------------
@@ -117,6 +121,7 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
         }
     tri_status st = TRI_OK;
     do {
+        if ((e = prepare_device()) != cudaSuccess) break;
         if ((e = cudaMalloc(&c->omega_d, sizeof omega)) != cudaSuccess) break;
         if ((e = cudaMalloc(&c->dbar_d, sizeof dbar)) != cudaSuccess) break;
         if ((e = cudaMalloc(&c->qc_d, nq * kHeadDim * sizeof(float))) != cudaSuccess) break;
@@ -259,6 +264,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, int32_t n_layers, CUtensorMap *out)
 {
     static EncodeTiledFn fn = nullptr;
+    static std::mutex fn_mu;
+    std::lock_guard<std::mutex> lock(fn_mu);
     if (!fn) {
         void *ptr = nullptr;
         cudaDriverEntryPointQueryResult q;
@@ -295,14 +302,40 @@ tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, 
     return TRI_OK;
 }
 
+// Opt-in shared-memory size of the scoring kernel.  The attribute belongs to (function, device); tri_create sets it
+// on the context's device, so contexts on several GPUs need no process-wide bookkeeping.
+template <int NT, int LAYOUT>
+cudaError_t allow_score_smem()
+{
+    return cudaFuncSetAttribute(k_score_tma<NT, LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreDynSmem);
+}
+
+cudaError_t prepare_device()
+{
+    cudaError_t e;
+    if ((e = allow_score_smem<1, 0>()) != cudaSuccess) return e;
+    if ((e = allow_score_smem<2, 0>()) != cudaSuccess) return e;
+    if ((e = allow_score_smem<4, 0>()) != cudaSuccess) return e;
+    if ((e = allow_score_smem<1, 1>()) != cudaSuccess) return e;
+    if ((e = allow_score_smem<2, 1>()) != cudaSuccess) return e;
+    return allow_score_smem<4, 1>();
+}
+
+// Every entry point that launches kernels runs on the device the context was created on.
+tri_status check_device(const tri_ctx *c)
+{
+    int dev = -1;
+    TRI_CUDA(cudaGetDevice(&dev));
+    if (dev != c->device) {
+        snprintf(g_err, sizeof g_err, "context belongs to device %d but device %d is current", c->device, dev);
+        return TRI_ERR_INVALID_ARG;
+    }
+    return TRI_OK;
+}
+
 template <int NT, int LAYOUT>
 tri_status launch_score_tma_one(dim3 grid, cudaStream_t st, const CUtensorMap &map, const ScoreParams &sp)
 {
-    static bool configured = false;
-    if (!configured) {
-        TRI_CUDA(cudaFuncSetAttribute(k_score_tma<NT, LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreDynSmem));
-        configured = true;
-    }
     k_score_tma<NT, LAYOUT><<<grid, kScoreThreads, kScoreDynSmem, st>>>(map, sp);
     return TRI_OK;
 }
@@ -374,12 +407,11 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
 // Top-B selection.  pl == NULL: from the final scores in `scores` (tri_select).  pl != NULL: the fused round,
 // straight from the raw scores and partial sums in the workspace `ws`; final scores are parked in its score area.
 tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
-                      int32_t budget, int32_t *kept_idx, int32_t *kept_cnt, int32_t *new_seq_lens,
+                      int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
                       int32_t U, const Plan *pl, char *ws, cudaStream_t st)
 {
     SelectParams p;
     p.scores = scores; p.scores_w = nullptr; p.seq_lens = seq_lens; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
-    p.new_seq_lens = new_seq_lens;
     p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget;
     p.raw = nullptr; p.partials = nullptr; p.G = c->desc.group_size; p.chunk = 0; p.nchunks = 0;
     if (pl) {
@@ -462,6 +494,7 @@ extern "C" tri_status tri_score(tri_ctx *c, const tri_cache_view *src, int32_t S
 {
     tri_status r;
     if (!c || !src || !cur_pos || !scores || !ws) return TRI_ERR_INVALID_ARG;
+    if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_view(src, true)) != TRI_OK) return r;
     if ((r = check_common(c, S, src->n_max, 1)) != TRI_OK) return r;
     if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
@@ -477,9 +510,10 @@ extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t 
     (void)ws; (void)ws_bytes;   // the selection keeps its histograms and candidates in shared memory
     tri_status r;
     if (!c || !scores || !seq_lens || !kept_idx || !kept_cnt) return TRI_ERR_INVALID_ARG;
+    if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_common(c, S, n_max, budget)) != TRI_OK) return r;
     int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
-    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, nullptr, U, nullptr, nullptr,
+    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, U, nullptr, nullptr,
                       (cudaStream_t)stream);
 }
 
@@ -489,6 +523,7 @@ extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const i
 {
     tri_status r;
     if (!c || !kept_idx || !kept_cnt) return TRI_ERR_INVALID_ARG;
+    if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_view(src, false)) != TRI_OK) return r;
     if ((r = check_view(dst, false)) != TRI_OK) return r;
     if ((r = check_common(c, S, src->n_max, budget)) != TRI_OK) return r;
@@ -518,12 +553,14 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
     }
     {
         NvtxRange part("tri_compress: normalise + select");
-        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, new_seq_lens, pl.U, &pl, w,
+        // new_seq_lens may be the very array the scoring and selection kernels read the lengths from, so only the
+        // last launch of the round (the gather, which reads kept counts, never lengths) stores it
+        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, pl.U, &pl, w,
                             st)) != TRI_OK)
             return r;
     }
     NvtxRange part("tri_compress: compact");
-    return run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, pl.U, st);
+    return run_compact(c, src, idx, cnt, S, budget, dst, new_seq_lens, device_status, pl.U, st);
 }
 
 extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
@@ -533,6 +570,7 @@ extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_
 {
     tri_status r;
     if (!c || !cur_pos || !ws) return TRI_ERR_INVALID_ARG;
+    if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_view(src, true)) != TRI_OK) return r;
     if ((r = check_view(dst, false)) != TRI_OK) return r;
     if ((r = check_common(c, S, src->n_max, budget)) != TRI_OK) return r;
@@ -567,6 +605,7 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
     if (!src_host->seq_lens || !src_dev->seq_lens || !src_host->k || !dst_host->k) return TRI_ERR_INVALID_ARG;
     tri_status r;
     NvtxRange whole("tri_compress_host");
+    if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_view(src_dev, true)) != TRI_OK) return r;
     if ((r = check_view(dst_dev, false)) != TRI_OK) return r;
     if ((r = check_common(c, S, src_dev->n_max, budget)) != TRI_OK) return r;
@@ -587,13 +626,15 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
     const bool sparse = 2 * (int64_t)budget <= src_dev->n_max;
     void *v_alias = (sparse && src_host->v && src_dev->v) ? device_alias(src_host->v) : nullptr;
     void *pos_alias = (sparse && src_host->positions && src_dev->positions) ? device_alias(src_host->positions) : nullptr;
-    TRI_CUDA(cudaMemcpyAsync((void *)src_dev->seq_lens, src_host->seq_lens, S * sizeof(int32_t),
-                             cudaMemcpyHostToDevice, st));
-    TRI_CUDA(cudaMemcpyAsync(cur_pos_dev, cur_pos_host, S * sizeof(int64_t), cudaMemcpyHostToDevice, st));
-
     // Layer ranges: range i is copied in and compressed on the caller's stream; its results go back to the host
     // on the context's copy stream while range i + 1 is already coming in (the link is full duplex).
     const int M = c->have_back ? (L < kHostSlabs ? L : kHostSlabs) : 1;
+    // the workspace must hold the largest range; checked before the first copy is enqueued
+    const int widest = (L + M - 1) / M;
+    if (ws_bytes < make_plan(c, S, src_dev->n_max, budget, widest).total) return TRI_ERR_WORKSPACE;
+    TRI_CUDA(cudaMemcpyAsync((void *)src_dev->seq_lens, src_host->seq_lens, S * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, st));
+    TRI_CUDA(cudaMemcpyAsync(cur_pos_dev, cur_pos_host, S * sizeof(int64_t), cudaMemcpyHostToDevice, st));
     cudaStream_t back = M > 1 ? c->back : st;
     const size_t upl = (size_t)S * H;                                  // units per layer
     for (int i = 0; i < M; ++i) {

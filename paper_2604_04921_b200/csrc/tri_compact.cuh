@@ -31,6 +31,17 @@ __device__ __forceinline__ uint4 ld_once(const void *p)
     return r;
 }
 
+// The same streaming load without the read-only (.nc) path: for kernels that later overwrite the buffer they read.
+__device__ __forceinline__ uint4 ld_stream(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p)
+                 : "memory");
+    return r;
+}
+
 __device__ __forceinline__ void st_once(void *p, uint4 v)
 {
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
@@ -93,7 +104,7 @@ __global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const Compact
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
             const int64_t o = __shfl_sync(0xffffffffu, so, r);
-            if (o >= 0) val[r] = ld_once(sb + o * 2);
+            if (o >= 0) val[r] = AFTER_PREFIX ? ld_stream(sb + o * 2) : ld_once(sb + o * 2);   // in place: no read-only path
         }
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
@@ -220,7 +231,7 @@ __global__ void __launch_bounds__(kInplaceThreads, 2) k_compact_inplace_rows(con
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
             const int64_t o = __shfl_sync(0xffffffffu, so, r);
-            if (o >= 0) val[r] = ld_once(sb + o * 2);
+            if (o >= 0) val[r] = ld_stream(sb + o * 2);
         }
         __syncthreads();                                     // every source of the tile has been read
 #pragma unroll
@@ -249,33 +260,38 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace_any(const C
 
     for (int j0 = 0; j0 < cnt; j0 += kInplaceAnyRows) {
         const int rows = min(kInplaceAnyRows, cnt - j0);
+        // a row moves only if its index is inside the unit and both addresses resolve; anything else is reported
+        // and left alone
+        auto source_of = [&](int r) -> int64_t {
+            const int srow = __ldg(idx + j0 + r);
+            if (srow == j0 + r) return -2;                     // already in its slot
+            return (srow >= 0 && srow < p.src.n_max) ? row_offset(p.src, l, s, h, srow) : -1;
+        };
         for (int i = threadIdx.x; i < rows * per_row; i += kInplaceThreads) {
-            int r = i / per_row, c = i - r * per_row;
-            int srow = __ldg(idx + j0 + r);
-            if (srow == j0 + r) continue;                      // already in its slot
-            int64_t so = (srow >= 0 && srow < p.src.n_max) ? row_offset(p.src, l, s, h, srow) : -1;
-            const bool is_k = c < p.k_vec;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (so < 0) { if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK); }
-            else v = is_k ? ld_once(p.src.k + so * p.k_esize + c * 16)
-                          : ld_once(p.src.v + so * 2 + (c - p.k_vec) * 16);
-            stage[i] = v;
+            const int r = i / per_row, c = i - r * per_row;
+            const int64_t so = source_of(r);
+            if (so == -1 && c == 0 && p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
+            if (so < 0) continue;
+            stage[i] = c < p.k_vec ? ld_stream(p.src.k + so * p.k_esize + c * 16)
+                                   : ld_stream(p.src.v + so * 2 + (c - p.k_vec) * 16);
         }
         if (p.dst.positions && threadIdx.x < rows) {
-            int srow = min(max(__ldg(idx + j0 + threadIdx.x), 0), p.src.n_max - 1);
-            pos_s[threadIdx.x] = p.src.positions ? p.src.positions[(int64_t)u * p.src.n_max + srow] : srow;
+            const int srow = __ldg(idx + j0 + threadIdx.x);
+            const bool ok = srow >= 0 && srow < p.src.n_max;
+            pos_s[threadIdx.x] = !ok ? -1 : (p.src.positions ? p.src.positions[(int64_t)u * p.src.n_max + srow] : srow);
         }
         __syncthreads();
         for (int i = threadIdx.x; i < rows * per_row; i += kInplaceThreads) {
-            int r = i / per_row, c = i - r * per_row;
-            if (__ldg(idx + j0 + r) == j0 + r) continue;
-            int64_t dof = row_offset(p.dst, l, s, h, j0 + r);
+            const int r = i / per_row, c = i - r * per_row;
+            if (source_of(r) < 0) continue;
+            const int64_t dof = row_offset(p.dst, l, s, h, j0 + r);
             const bool is_k = c < p.k_vec;
             if (dof < 0) { if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK); }
             else if (is_k) *reinterpret_cast<uint4 *>(p.dst.k + dof * p.k_esize + c * 16) = stage[i];
             else *reinterpret_cast<uint4 *>(p.dst.v + dof * 2 + (c - p.k_vec) * 16) = stage[i];
         }
-        if (p.dst.positions && threadIdx.x < rows)
+        if (p.dst.positions && threadIdx.x < rows && pos_s[threadIdx.x] >= 0 &&
+            __ldg(idx + j0 + threadIdx.x) != j0 + (int)threadIdx.x)
             p.dst.positions[(int64_t)u * p.dst.n_max + j0 + threadIdx.x] = pos_s[threadIdx.x];
         __syncthreads();
     }

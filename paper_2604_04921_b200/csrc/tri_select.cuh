@@ -33,7 +33,6 @@ struct SelectParams {
     const int32_t *seq_lens;  // [S]
     int32_t *kept_idx;        // [U][budget]
     int32_t *kept_cnt;        // [U]
-    int32_t *new_seq_lens;    // [S] or NULL
     int32_t S, H, n_max, budget;
     // FUSED only: raw scores and partial sums of the scoring kernel
     const float *raw;         // [U][n_max][G]
@@ -118,10 +117,7 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
     const float *sc = p.scores + (int64_t)u * p.n_max;
     int32_t *out = p.kept_idx + (int64_t)u * p.budget;
     const int cnt = min(n, p.budget);
-    if (tid == 0) {
-        p.kept_cnt[u] = cnt;
-        if (p.new_seq_lens && (u % p.H) == 0 && u / (p.H * p.S) == 0) p.new_seq_lens[s] = cnt;
-    }
+    if (tid == 0) p.kept_cnt[u] = cnt;
     if (n <= p.budget) {                        // the cache does not exceed the budget: keep all
         for (int i = tid; i < n; i += kSelThreads) out[i] = i;
         return;

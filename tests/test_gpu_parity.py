@@ -293,6 +293,44 @@ def test_decode_windows_in_place_over_several_rounds():
             host[h] = dict(k=kk[sel], v=vv[sel], pos=want_pos)
 
 
+def test_lengths_updated_in_place_with_many_units():
+    """new_seq_lens may be the array the round reads its lengths from (a decode loop updating them in place).
+    With far more units than one wave of thread blocks, every unit must still see the old length: a length
+    stored early by one block would make the later blocks of that sequence keep rows 0..B-1 instead of the top B."""
+    sp = W.SPECS["qwen3_8b_steady_b64"].scaled(name="alias", n_layers=8, n_kv_heads=8, n_seqs=64, n_keys=400, budget=256,
+                                               n_new=144, pos_lo=400, pos_hi=4000)
+    w = W.make_workload(sp, DEV)
+    B, S, H, L = sp.budget, sp.n_seqs, sp.n_kv_heads, sp.n_layers
+    lens0 = torch.randint(300, 401, (S,), dtype=torch.int32, device=DEV, generator=torch.Generator(DEV).manual_seed(7))
+    w.seq_lens = lens0.clone()
+    ctx = make_ctx(w)
+    src = src_view(w)
+    U = L * S * H
+    ws = ctx.workspace(S, sp.n_keys, B)
+    ref_idx = torch.full((U, B), -1, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(U, dtype=torch.int32, device=DEV)
+    k2 = torch.zeros(L, S, H, B, 128, dtype=torch.bfloat16, device=DEV); v2 = torch.zeros_like(k2)
+    p2 = torch.zeros(L, S, H, B, dtype=torch.int32, device=DEV)
+    dst = tb.CacheView(k2, v2, positions=p2)
+    separate = torch.zeros(S, dtype=torch.int32, device=DEV)
+    ctx.compress(src, w.cur_pos, B, dst, ws, kept_idx=ref_idx, kept_cnt=cnt, new_seq_lens=separate)
+    torch.cuda.synchronize()
+    assert separate.tolist() == [B] * S and w.seq_lens.tolist() == lens0.tolist()
+    for rep in range(3):                                   # aliased: three times, the race was timing dependent
+        w.seq_lens.copy_(lens0)
+        idx = torch.full((U, B), -1, dtype=torch.int32, device=DEV)
+        ctx.compress(src, w.cur_pos, B, dst, ws, kept_idx=idx, kept_cnt=cnt, new_seq_lens=w.seq_lens)
+        torch.cuda.synchronize()
+        assert w.seq_lens.tolist() == [B] * S
+        assert torch.equal(idx, ref_idx), rep
+    keep_all = torch.arange(B, dtype=torch.int32, device=DEV)
+    assert not bool((ref_idx == keep_all).all(dim=1).any())      # no unit took the keep-everything path
+    w.seq_lens.copy_(lens0)
+    res = dict(kept_idx=ref_idx, kept_cnt=cnt, k_out=k2, v_out=v2, pos_out=p2)
+    for (l, s, h) in [(0, 0, 0), (3, 17, 5), (7, 63, 7), (5, 40, 2)]:
+        check_unit(w, res, oracle_unit(w, l, s, h, B), l, s, h, B)
+
+
 def test_only_overflowing_sequences_are_touched():
     """A batch in which one sequence exceeds the budget and two do not: the short ones are kept whole, in order,
     and the round gives the same kept rows for the long one as a batch holding it alone."""
@@ -459,6 +497,34 @@ def test_bad_page_id_sets_status_not_fault():
     w.page_table[0, 3] = 10 ** 6
     res = run_compress(w, sp.budget, want_scores=False)
     assert int(res["status"].item()) == 5
+
+
+@pytest.mark.parametrize("fp32_keys", [True, False])
+def test_out_of_range_kept_index_is_skipped_in_place(fp32_keys):
+    """tri_compact in place with a kept index beyond the unit's capacity: that row is left as it was (not
+    overwritten, not dereferenced); every other row moves.  fp32 keys without a value cache take the staged
+    in-place kernel, bf16 K + V the tiled one."""
+    n, cnt = 96, 40
+    g = torch.Generator().manual_seed(11)
+    k = torch.randn(1, 1, 1, n, 128, generator=g).to(DEV)
+    if not fp32_keys:
+        k = k.to(torch.bfloat16)
+    v = None if fp32_keys else torch.randn(1, 1, 1, n, 128, generator=g).to(DEV).to(torch.bfloat16)
+    pos = torch.arange(100, 100 + n, dtype=torch.int32, device=DEV).view(1, 1, 1, n)
+    k0, pos0 = k.clone(), pos.clone()
+    idx = torch.arange(cnt, dtype=torch.int32) * 2 + 1           # 1, 3, 5, ...: ascending, idx[j] > j
+    idx[-1] = 10 ** 6
+    idx_d = idx.view(1, cnt).to(DEV)
+    cnt_d = torch.tensor([cnt], dtype=torch.int32, device=DEV)
+    ctx = tb.TriContext(1, 1, 1, torch.zeros(1, 1, 128), torch.zeros(1, 1, 64))
+    view = tb.CacheView(k, v, positions=pos)
+    ctx.compact(view, idx_d, cnt_d, 1, cnt, view)
+    torch.cuda.synchronize()
+    good = idx[:-1].long().to(DEV)
+    assert torch.equal(k[0, 0, 0, :cnt - 1], k0[0, 0, 0][good])
+    assert torch.equal(pos[0, 0, 0, :cnt - 1], pos0[0, 0, 0][good])
+    assert torch.equal(k[0, 0, 0, cnt - 1:], k0[0, 0, 0, cnt - 1:])          # the bad row and everything behind it
+    assert torch.equal(pos[0, 0, 0, cnt - 1:], pos0[0, 0, 0, cnt - 1:])
 
 
 def test_bounded_wait_runs_out_and_reports():
