@@ -6,13 +6,19 @@
 One step = one pass of the whole hot path (phasor fold, scoring, z-score/max, top-B select, gather
 compaction) over every (sequence, layer, KV head) unit of the workload.  Prints ONE JSON line.
 
-* value      keys scored+selected+compacted per second, inputs resident in HBM, CUDA events around K
-             steps, max over ranks (N > 1: independent replicas, one per GPU, "weak" scaling).
-* e2e        the same metric through tri_compress_host: pinned host K/V in, compacted K/V out, copies
-             inside the timed region.
-* roofline   the scoring kernel (it streams the whole key cache): algorithmic bytes / its mean launch
-             time, measured with CUDA events recorded by the library between its launches in a second
-             pass of K steps.
+* value       keys scored+selected+compacted per second on the headline workload (the 131,072-token
+              sequence unless --workload says otherwise), inputs resident in HBM, CUDA events around exactly
+              K steps, max over ranks (N > 1: independent replicas, one per GPU, "weak" scaling).
+* sustained   the same workload run back to back for about one second (the power-capped regime), with the
+              clock samples of that second.
+* workloads   at N = 1 and without --workload: the other benchmark configurations (steady-state batch,
+              32K one-shot, a 16-layer slab of the ragged paged batch) timed the same way, each with its
+              achieved fraction of the HBM roofline.
+* e2e         the headline metric through tri_compress_host: pinned host K/V in, compacted K/V out, copies
+              inside the timed region.
+* roofline    the scoring kernel (it streams the whole key cache): algorithmic bytes / its mean launch
+              time, measured with CUDA events recorded by the library around its launches in a second
+              pass of K steps.
 * cpu_baseline  the float64 oracle, as it stands, on a bounded sample of units of the same workload.
 
 --impl reference times that oracle alone (rank 0 only), one sampled unit per step.
@@ -31,12 +37,14 @@ if ROOT not in sys.path:
 
 METRIC = "tri_compress keys scored+selected+compacted per sec"
 UNIT = "keys/s"
-DEFAULT_WORKLOAD = "qwen3_8b_oneshot_32k"
+DEFAULT_WORKLOAD = "qwen3_8b_long_128k"
+# the other configurations a default run also times: (workload, layers; 0 = all)
+OTHER_WORKLOADS = (("qwen3_8b_steady_b64", 0), ("qwen3_8b_oneshot_32k", 0), ("qwen3_32b_ragged_paged", 16))
 NOMINAL_HBM_GBS = 8000.0
 
 
-# DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum on
-# 1,048,576 keys: 268.564992 MB + 13.988352 MB), valid only for the kernel source it was taken on.
+# DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum per key),
+# valid only for the kernel source it was taken on.
 SCORE_TRAFFIC = {"bytes_per_key": (268564992 + 13988352) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
@@ -59,17 +67,18 @@ def measured_peaks():
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except Exception:
-        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return 6650.0, "fallback (6.65 TB/s, an earlier measurement on B200)"
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi for the life of the run; a timed region asks for
+    the samples that fell between its mark() and its summary()."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc, self.first = index, [], None, 0
+        self.index, self.rows, self.proc = index, [], None
 
     def start(self):
         """Starts nvidia-smi and waits for its first sample: its start-up can stall the GPU for seconds and
@@ -86,28 +95,25 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def mark(self):
-        """Samples taken from now on count (call right before the timed region)."""
-        self.first = len(self.rows)
-
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
-    def stop(self):
+    def mark(self):
+        """Index of the next sample (call right before a timed region)."""
+        return len(self.rows)
+
+    def summary(self, first: int):
+        """Median SM clock and active throttle reasons of the samples taken since mark() returned `first`."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.06)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
+        last = len(self.rows)
+        # a timed region shorter than the sampling period holds no sample: fall back to the whole run so far
+        window = "timed region" if last > first else "whole run so far (timed region shorter than one sample)"
+        rows = self.rows[first:last] if last > first else self.rows[:last]
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        # a timed region shorter than the sampling period holds no sample: fall back to the whole run
-        window = "timed region" if len(self.rows) > self.first else "whole run (timed region shorter than one sample)"
-        rows = self.rows[self.first:] if len(self.rows) > self.first else self.rows
         for r in rows:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
@@ -120,6 +126,15 @@ class ClockSampler:
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "samples": len(sm), "window": window, "reasons": sorted(reasons)}
 
+    def stop(self):
+        if self.proc is None:
+            return
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+
 
 def algorithmic_bytes(seq_lens, units_per_seq, budget):
     """256 N (stream K) + 1036 min(B, N) (re-read kept K, read kept V, write both, idx + positions)."""
@@ -127,6 +142,19 @@ def algorithmic_bytes(seq_lens, units_per_seq, budget):
     for n in seq_lens:
         tot += units_per_seq * (256 * n + 1036 * min(budget, n))
     return tot
+
+
+def workload_config(spec, L, world=1):
+    """The `config` object of the JSON line; both arms (the CUDA path and --impl reference) print the same one."""
+    S, H = spec.n_seqs, spec.n_kv_heads
+    return {"workload": spec.name + (f"[first {L} layers]" if L != spec.n_layers else ""),
+            "units": L * S * H, "layers": L, "kv_heads": H, "group_size": spec.group_size, "seqs": S,
+            "keys_per_unit": spec.n_keys if spec.kind != "ragged_paged" else f"{spec.n_keys_min}..{spec.n_keys}",
+            "budget": spec.budget, "storage_dtype": "bf16", "accumulate_dtype": "f32", "paged": spec.kind == "ragged_paged",
+            "compaction": "in place into the sequence's pages, pool restored between steps outside the timed region"
+            if spec.kind == "ragged_paged" else "out of place",
+            "l2": "inputs larger than L2 (GB of K+V per step in hbm.kv_bytes)",
+            "parallelism": "replicas" if world > 1 else "single GPU"}
 
 
 def oracle_sample(spec, units, budget):
@@ -189,18 +217,18 @@ def run_reference(args, spec):
     if args.steps <= 0:
         args.steps = 4
     oracle.build()
-    units = sample_units(spec, args.warmup + args.steps)
-    oracle_sample(spec, units[:max(1, min(args.warmup, 1))], spec.budget)     # warm-up: page in, build
-    keys, secs = oracle_sample(spec, units[args.warmup:args.warmup + args.steps], spec.budget)
+    L = args.layers if args.layers > 0 else spec.n_layers
+    units = sample_units(spec.scaled(n_layers=L), 1 + args.steps)
+    oracle_sample(spec, units[:1], spec.budget)                      # warm-up: page in, build
+    keys, secs = oracle_sample(spec, units[1:1 + args.steps], spec.budget)
     val = keys / secs
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": spec.name, "units_per_step": 1, "keys_per_unit": spec.n_keys,
-                       "budget": spec.budget},
+            "config": workload_config(spec, L),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                             "sample": f"{args.steps} units of {spec.n_keys} keys (one per step) out of "
-                                       f"{spec.n_layers * spec.n_seqs * spec.n_kv_heads}"},
+                             "sample": f"each step = one unit of the workload, {args.steps} units ({keys} keys) out of "
+                                       f"{L * spec.n_seqs * spec.n_kv_heads}; one untimed warm-up unit"},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -216,7 +244,7 @@ def run_calibration(args):
     torch.cuda.set_device(0)
     tb.lib()
     sp = W.SPECS["qwen3_8b_oneshot_32k"]
-    T, Hq = 262144, sp.n_kv_heads * sp.group_size
+    T, Hq = (args.tokens if args.tokens > 0 else 262144), sp.n_kv_heads * sp.group_size
     q = W.make_queries(sp, 0, T, "cuda", dtype=torch.bfloat16)
     cal = tb.Calibrator(Hq)
     for _ in range(max(3, args.warmup)):
@@ -254,17 +282,117 @@ def run_calibration(args):
     print(json.dumps(line), flush=True)
 
 
+class Round:
+    """One workload resident on the device with everything a timed tri_compress step needs."""
+
+    def __init__(self, spec, L, dev):
+        import torch
+        from paper_2604_04921_b200 import binding as tb
+        from paper_2604_04921_b200 import workloads as W
+        self.spec, self.L, self.dev = spec, L, dev
+        self.w = w = W.make_workload(spec, dev, layer0=0, n_layers=L)
+        S, H, G, B = spec.n_seqs, spec.n_kv_heads, spec.group_size, spec.budget
+        self.ctx = tb.TriContext(L, H, G, w.q_center, w.q_mean_norm, rope_theta=spec.theta)
+        self.src = tb.CacheView(w.k, w.v, seq_lens=w.seq_lens, positions=w.positions, page_table=w.page_table)
+        self.n_max = self.src.c_view().n_max
+        self.U = L * S * H
+        if w.paged:
+            # compacted rows are written back into the sequence's own pages (in place)
+            self.dst = tb.CacheView(w.k, w.v, page_table=w.page_table, n_max=self.n_max)
+            self.k2 = self.v2 = self.p2 = None
+        else:
+            self.k2 = torch.empty(L, S, H, B, 128, dtype=torch.bfloat16, device=dev)
+            self.v2 = torch.empty_like(self.k2)
+            self.p2 = torch.empty(L, S, H, B, dtype=torch.int32, device=dev)
+            self.dst = tb.CacheView(self.k2, self.v2, positions=self.p2)
+        self.ws = self.ctx.workspace(S, self.n_max, B, dev)
+        self.kept_cnt = torch.zeros(self.U, dtype=torch.int32, device=dev)
+        self.lens = w.seq_lens.tolist()
+        self.keys_per_step = sum(self.lens) * L * H
+        self.abytes = algorithmic_bytes(self.lens, L * H, B)
+        self.launches_per_step = self.ctx.compress_launches(self.src, S, self.dst)
+        # An in-place round changes its own input (the kept rows move to the front of each sequence's pages), and
+        # a second round on that state would find nearly every kept row already in place.  So for the paged
+        # workload every step starts from the pristine pool: the pages a round overwrites are put back from a copy
+        # between steps, outside the timed region, and each step is timed on its own.
+        self.restore = None
+        if w.paged:
+            ps = spec.page_size
+            keep_pages = (B + ps - 1) // ps
+            pages = torch.cat([w.page_table[s, :min(keep_pages, (self.lens[s] + ps - 1) // ps)] for s in range(S)]).long()
+            k_bak, v_bak = w.k[:, pages].clone(), w.v[:, pages].clone()
+
+            def restore():
+                w.k[:, pages] = k_bak
+                w.v[:, pages] = v_bak
+            self.restore = restore
+
+    def step(self):
+        self.ctx.compress(self.src, self.w.cur_pos, self.spec.budget, self.dst, self.ws, kept_cnt=self.kept_cnt)
+
+    def timed_steps(self, n):
+        """n steps; returns their total device time in ms (this rank)."""
+        import torch
+        if self.restore is None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                self.step()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+        evs = []
+        for _ in range(n):
+            self.restore()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            self.step()
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in evs)
+
+    def warm(self, n):
+        for _ in range(n):
+            if self.restore is not None:
+                self.restore()
+            self.step()
+
+    def kernel_ms(self, steps):
+        """Mean duration of each kernel kind per step: events recorded by the library around its launches."""
+        self.ctx.profile_begin()
+        per = {k: 0.0 for k in self.ctx.KERNELS}
+        for _ in range(steps):
+            if self.restore is not None:
+                self.restore()
+            self.step()
+            for k, v in self.ctx.profile_read().items():
+                per[k] += v / steps
+        self.ctx.profile_end()
+        return per
+
+    def hbm(self, ms_step, peak):
+        gbs = self.abytes / (ms_step * 1e-3) / 1e9
+        return {"algorithmic_bytes_per_step": self.abytes, "kv_bytes": (self.w.k.numel() + self.w.v.numel()) * 2,
+                "achieved_gbs": gbs, "frac_of_measured_copy_peak": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS}
+
+    def close(self):
+        self.ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=0, help="timed steps; 0 = as many as fill about one second")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--workload", default=None, help=f"headline workload (default {DEFAULT_WORKLOAD}, plus the others)")
     ap.add_argument("--layers", type=int, default=0, help="only the first LAYERS layers (a slab); 0 = all")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="time the headline workload only")
     ap.add_argument("--calibration", action="store_true", help="time the calibration-statistics pass instead of the round")
+    ap.add_argument("--tokens", type=int, default=0, help="--calibration: tokens per pass (default 262,144)")
     args = ap.parse_args()
     if args.calibration:
         run_calibration(args)
@@ -272,7 +400,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
     from paper_2604_04921_b200 import workloads as W
-    spec = W.SPECS[args.workload]
+    others = args.workload is None and args.layers == 0 and not args.no_others
+    spec = W.SPECS[args.workload or DEFAULT_WORKLOAD]
     if args.impl == "reference":
         run_reference(args, spec)
         return
@@ -293,140 +422,78 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     tb.lib()   # fails loudly if the CUDA library has not been built
 
-    L = args.layers if args.layers > 0 else spec.n_layers
-    w = W.make_workload(spec, dev, layer0=0, n_layers=L)
-    S, H, G, B = spec.n_seqs, spec.n_kv_heads, spec.group_size, spec.budget
-    ctx = tb.TriContext(L, H, G, w.q_center, w.q_mean_norm, rope_theta=spec.theta)
-    src = tb.CacheView(w.k, w.v, seq_lens=w.seq_lens, positions=w.positions, page_table=w.page_table)
-    n_max = src.c_view().n_max
-    U = L * S * H
-    if w.paged:
-        # compacted rows are written back into the sequence's own pages (in place)
-        dst = tb.CacheView(w.k, w.v, page_table=w.page_table, n_max=n_max)
-    else:
-        k2 = torch.empty(L, S, H, B, 128, dtype=torch.bfloat16, device=dev)
-        v2 = torch.empty_like(k2)
-        p2 = torch.empty(L, S, H, B, dtype=torch.int32, device=dev)
-        dst = tb.CacheView(k2, v2, positions=p2)
-    ws = ctx.workspace(S, n_max, B, dev)
-    kept_cnt = torch.zeros(U, dtype=torch.int32, device=dev)
-    lens = w.seq_lens.tolist()
-    keys_per_step = sum(lens) * L * H
-    abytes = algorithmic_bytes(lens, L * H, B)
-    launches_per_step = ctx.compress_launches(src, dst)
-
-    def step():
-        ctx.compress(src, w.cur_pos, B, dst, ws, kept_cnt=kept_cnt)
-
     def barrier():
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # An in-place round changes its own input (the kept rows move to the front of each sequence's pages), and
-    # a second round on that state would find nearly every kept row already in place.  So for the paged
-    # workload every step starts from the pristine pool: the pages a round overwrites are put back from a copy
-    # between steps, outside the timed region, and each step is timed on its own.
-    restore = None
-    if w.paged:
-        ps = spec.page_size
-        keep_pages = (B + ps - 1) // ps
-        pages = torch.cat([w.page_table[s, :min(keep_pages, (lens[s] + ps - 1) // ps)] for s in range(S)]).long()
-        k_bak, v_bak = w.k[:, pages].clone(), w.v[:, pages].clone()
-
-        def restore():
-            w.k[:, pages] = k_bak
-            w.v[:, pages] = v_bak
-
-    def timed_steps(n):
-        """n steps; returns their total device time in ms (this rank)."""
-        if restore is None:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(n):
-                step()
-            e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1)
-        evs = []
-        for _ in range(n):
-            restore()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            step()
-            e1.record()
-            evs.append((e0, e1))
-        torch.cuda.synchronize()
-        return sum(a.elapsed_time(b) for a, b in evs)
-
+    peak, peak_src = measured_peaks()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    for _ in range(args.warmup):
-        if restore is not None:
-            restore()
-        step()
-    barrier()
-    if args.steps <= 0:
-        # fill about one second, so that the clock sampler sees the region under load
-        est = max_over_ranks(timed_steps(3) / 3, dist, dev)
+
+    def second_of_steps(rd):
+        """About one second of back-to-back steps (the power-capped regime) with its clock samples."""
+        est = max_over_ranks(rd.timed_steps(3) / 3, dist, dev)
         barrier()
-        args.steps = int(min(3000, max(20, 1000.0 / est)))
-    sampler.mark()
-    ms_mine = timed_steps(args.steps)
+        n = int(min(3000, max(20, 1000.0 / est)))
+        first = sampler.mark()
+        ms = max_over_ranks(rd.timed_steps(n), dist, dev) / n
+        barrier()
+        return n, ms, (sampler.summary(first) if rank == 0 else None)
+
+    L = args.layers if args.layers > 0 else spec.n_layers
+    rd = Round(spec, L, dev)
+    rd.warm(args.warmup)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    ms_step = max_over_ranks(ms_mine, dist, dev) / args.steps
+    sustained = None
+    if args.steps <= 0:
+        args.steps, ms_step, clocks = second_of_steps(rd)
+    else:
+        first = sampler.mark()
+        ms_step = max_over_ranks(rd.timed_steps(args.steps), dist, dev) / args.steps
+        barrier()
+        clocks = sampler.summary(first) if rank == 0 else None
+        n, ms, ck = second_of_steps(rd)
+        sustained = {"steps": n, "ms_per_step": ms, "value": whole_job_value(world, rd.keys_per_step, ms), "unit": UNIT,
+                     "hbm": rd.hbm(ms, peak), "clocks": ck}
 
-    # per-kernel durations: second pass, events recorded by the library between its launches
-    ctx.profile_begin()
-    per = {k: 0.0 for k in ctx.KERNELS}
-    prof_steps = min(args.steps, 200)
-    for _ in range(prof_steps):
-        if restore is not None:
-            restore()
-        step()
-        for k, v in ctx.profile_read().items():
-            per[k] += v / prof_steps
-    ctx.profile_end()
-
-    peak, peak_src = measured_peaks()
-    score_bytes = 256 * keys_per_step
+    per = rd.kernel_ms(min(args.steps, 50))
+    score_bytes = 256 * rd.keys_per_step
     score_gbs = score_bytes / (per["score"] * 1e-3) / 1e9
+    cfg = workload_config(spec, L, world)
     line = {
-        "metric": METRIC, "value": whole_job_value(world, keys_per_step, ms_step), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_value(world, rd.keys_per_step, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": spec.name + (f"[first {L} layers]" if L != spec.n_layers else ""),
-                   "units": U, "layers": L, "kv_heads": H, "group_size": G, "seqs": S, "keys_per_step": keys_per_step,
-                   "budget": B, "storage_dtype": "bf16", "paged": bool(w.paged),
-                   "compaction": "in place into the sequence's pages, pool restored between steps outside the timed region"
-                   if w.paged else "out of place",
-                   "l2": f"inputs larger than L2: {(w.k.numel() + w.v.numel()) * 2 / 1e9:.2f} GB of K+V read per step",
-                   "parallelism": "replicas" if world > 1 else "single GPU"},
-        "hbm": {"algorithmic_bytes_per_step": abytes, "achieved_gbs": abytes / (ms_step * 1e-3) / 1e9,
-                "frac_of_measured_copy_peak": abytes / (ms_step * 1e-3) / 1e9 / peak,
-                "frac_of_nominal_8tbs": abytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": cfg,
+        "keys_per_step": rd.keys_per_step,
+        "hbm": rd.hbm(ms_step, peak),
         "roofline": {"kernel": "k_score_tma", "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(keys_per_step), "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"]},
+                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(rd.keys_per_step), "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"],
+                     "note": "per step; a pipelined round issues the scoring as several launches over unit ranges, "
+                             "their bytes and durations are summed"},
         "kernel_ms": per,
-        "gpu_launches": launches_per_step * args.steps,
+        "gpu_launches": rd.launches_per_step * args.steps,
         "clocks": clocks,
     }
+    if sustained is not None:
+        line["sustained"] = sustained
 
     # ---- end to end through tri_compress_host: pinned host buffers, copies inside the timed region ----
+    w, S, B, U = rd.w, spec.n_seqs, spec.budget, rd.U
     if not args.no_e2e and not w.paged:
-        e2e_steps = max(2, min(args.steps, 5))
+        e2e_steps = max(2, min(args.steps, 3 if rd.keys_per_step > 2e7 else 5))
         hk = torch.empty(w.k.shape, dtype=w.k.dtype, pin_memory=True).copy_(w.k)
         hv = torch.empty(w.v.shape, dtype=w.v.dtype, pin_memory=True).copy_(w.v)
         hpos = None if w.positions is None else torch.empty(w.positions.shape, dtype=torch.int32, pin_memory=True).copy_(w.positions)
         hlens = torch.empty(S, dtype=torch.int32, pin_memory=True).copy_(w.seq_lens)
         hcur = torch.empty(S, dtype=torch.int64, pin_memory=True).copy_(w.cur_pos)
-        hk2 = torch.empty(k2.shape, dtype=k2.dtype, pin_memory=True)
-        hv2 = torch.empty(k2.shape, dtype=k2.dtype, pin_memory=True)
-        hp2 = torch.empty(p2.shape, dtype=torch.int32, pin_memory=True)
+        hk2 = torch.empty(rd.k2.shape, dtype=rd.k2.dtype, pin_memory=True)
+        hv2 = torch.empty(rd.k2.shape, dtype=rd.k2.dtype, pin_memory=True)
+        hp2 = torch.empty(rd.p2.shape, dtype=torch.int32, pin_memory=True)
         hcnt = torch.empty(U, dtype=torch.int32, pin_memory=True)
         dlens = torch.empty_like(w.seq_lens)
         dcur = torch.empty_like(w.cur_pos)
@@ -435,7 +502,7 @@ def main():
         dst_h = tb.CacheView(hk2, hv2, positions=hp2)
 
         def step_host():
-            ctx.compress_host(src_h, src_d, hcur, dcur, B, dst_h, dst, hcnt, kept_cnt, ws)
+            rd.ctx.compress_host(src_h, src_d, hcur, dcur, B, dst_h, rd.dst, hcnt, rd.kept_cnt, rd.ws)
 
         step_host()
         barrier()
@@ -446,19 +513,19 @@ def main():
         e1.record()
         barrier()
         ms_e2e = max_over_ranks(e0.elapsed_time(e1), dist, dev) / e2e_steps
-        assert int(hcnt.min()) == min(B, min(lens))
+        assert int(hcnt.min()) == min(B, min(rd.lens))
         # K is copied in full; of V and the positions only the kept rows cross the link (read by the gather
         # straight from the pinned host arrays)
-        kept_rows = sum(min(B, n) for n in lens) * L * H
-        if 2 * B <= n_max:
+        kept_rows = sum(min(B, n) for n in rd.lens) * L * spec.n_kv_heads
+        if 2 * B <= rd.n_max:
             h2d = hk.numel() * 2 + kept_rows * 256 + (0 if hpos is None else kept_rows * 4) + S * 12
         else:       # most rows are kept: V and positions are staged in bulk like K
             h2d = (hk.numel() + hv.numel()) * 2 + (0 if hpos is None else hpos.numel() * 4) + S * 12
         d2h = (hk2.numel() + hv2.numel()) * 2 + hp2.numel() * 4 + U * 4
-        line["e2e"] = {"value": whole_job_value(world, keys_per_step, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
+        line["e2e"] = {"value": whole_job_value(world, rd.keys_per_step, ms_e2e), "unit": UNIT, "ms_per_step": ms_e2e,
                        "steps": e2e_steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                        "call": "tri_compress_host (pinned host K/V/positions in, compacted K/V/positions/counts out; V and positions of kept rows read in place)"}
-        del hk, hv, hk2, hv2
+        del hk, hv, hk2, hv2, hpos, hp2, src_h, dst_h
     else:
         line["e2e"] = None
 
@@ -466,8 +533,9 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         oracle.build()
-        if restore is not None:
-            restore()
+        if rd.restore is not None:
+            rd.restore()
+        G = spec.group_size
         units = sample_units(spec.scaled(n_layers=L), 512)
         keys = secs = 0.0
         used = 0
@@ -486,6 +554,39 @@ def main():
                 break
         line["cpu_baseline"] = {"value": keys / secs, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                                 "sample": f"{used} of {U} units ({int(keys)} keys), oracle time {secs:.1f} s"}
+
+    # ---- the other benchmark configurations, same method (N = 1, default run only) ----
+    if others and world == 1:
+        rd.close()
+        del rd, w
+        torch.cuda.empty_cache()
+        entries = [{"workload": cfg["workload"], "steps": (sustained or {}).get("steps", args.steps),
+                    "ms_per_step": (sustained or {}).get("ms_per_step", ms_step),
+                    "value": (sustained or {}).get("value", line["value"]), "unit": UNIT,
+                    "hbm": (sustained or {}).get("hbm", line["hbm"]), "kernel_ms": per,
+                    "clocks": (sustained or {}).get("clocks", clocks), "burst_ms_per_step": ms_step, "burst_steps": args.steps}]
+        for name, layers in OTHER_WORKLOADS:
+            if name == spec.name:
+                continue
+            sp = W.SPECS[name]
+            Lo = layers if layers > 0 else sp.n_layers
+            r2 = Round(sp, Lo, dev)
+            r2.warm(3)
+            torch.cuda.synchronize()
+            first = sampler.mark()
+            burst = r2.timed_steps(20) / 20
+            n, ms, ck = second_of_steps(r2)
+            entries.append({"workload": workload_config(sp, Lo)["workload"], "steps": n, "ms_per_step": ms,
+                            "value": r2.keys_per_step / (ms * 1e-3), "unit": UNIT, "hbm": r2.hbm(ms, peak),
+                            "kernel_ms": r2.kernel_ms(min(n, 20)), "clocks": ck, "burst_ms_per_step": burst, "burst_steps": 20,
+                            "units": r2.U, "keys_per_step": r2.keys_per_step})
+            r2.close()
+            del r2
+            torch.cuda.empty_cache()
+        line["workloads"] = entries
+
+    if rank == 0:
+        sampler.stop()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

@@ -211,14 +211,38 @@ tri_status tri_compress_host(tri_ctx *ctx, const tri_cache_view *src_host, const
 tri_status tri_score_static(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                             float *scores, float *raw, void *stream);
 
-/* Number of kernel launches one tri_compress call issues for this shape (for launch accounting). */
-int32_t tri_compress_launches(const tri_ctx *ctx, const tri_cache_view *src, const tri_cache_view *dst);
+/*
+ * How tri_compress is issued (the paper has no counterpart; a scheduling choice of this library).
+ *   ranges = 1   every kernel of the round on the caller's stream, one launch each.
+ *   ranges > 1   the units are cut into that many contiguous ranges (at most 16).  The caller's stream scores range
+ *                after range; selection and compaction of a range run on a high-priority stream owned by the context
+ *                while the next range is being scored, so the latency-bound selection overlaps the key stream.  The
+ *                caller's stream waits for that stream before tri_compress returns control to it: work enqueued on
+ *                `stream` afterwards sees the finished round, and a stream capture sees the side stream joined.
+ *   ranges = 0   (default) chosen per call: about one range per 32 units, at most 8.
+ * Results are bit-identical in every mode.  One context must not run two tri_compress calls concurrently.
+ */
+tri_status tri_set_pipeline(tri_ctx *ctx, int32_t ranges);
+
+/*
+ * Which kernel scores bf16 keys (the paper has no counterpart; both compute the same Sections 4.1-4.2 scores to
+ * fp32 rounding, so results may differ in the last bits between the two, never within one):
+ *   0 (default)  tcgen05: 128-key tiles, tensor-memory accumulator, magnitudes staged through shared memory
+ *   1            mma.sync: 16-key warp tiles, everything in registers
+ * Call it before tri_workspace_bytes: the workspace layout depends on the kernel's block size.
+ */
+tri_status tri_set_score_kernel(tri_ctx *ctx, int32_t which);
+
+/* Number of kernel launches one tri_compress call issues for this shape and mode (for launch accounting). */
+int32_t tri_compress_launches(const tri_ctx *ctx, const tri_cache_view *src, int32_t S, const tri_cache_view *dst);
 
 /*
  * Measurement aid (the paper has no counterpart): between tri_profile_begin and tri_profile_end every
- * tri_compress call records a CUDA event before and after each of its 5 kernels (phasor fold, raw
- * scoring, z-score/max, top-B select, gather) on its stream.  tri_profile_read waits for the last
- * call's final event and writes the 5 kernel durations in milliseconds to ms[0..4] (host).
+ * tri_compress call records a CUDA event before and after each of its launches, on the stream the launch
+ * goes to.  tri_profile_read waits for the last call's events and writes the summed durations per kind of
+ * kernel in milliseconds to ms[0..4] (host): phasor fold, raw scoring, z-score/max (0 in the fused round,
+ * whose selection normalises), top-B select, gather.  In a pipelined round kernels of different kinds overlap,
+ * so the five figures may add up to more than the round took.
  * tri_profile_begin creates the events; it is the only one of the three that allocates.
  */
 tri_status tri_profile_begin(tri_ctx *ctx);

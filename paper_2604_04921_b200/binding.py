@@ -20,11 +20,11 @@ _ROOT = _PKG.parent
 LIB_PATH = _PKG / "lib" / "libtriattn.so"
 SOURCES = [_PKG / "csrc" / "tri_api.cu"]
 HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cuh", _PKG / "csrc" / "tri_score.cuh",
-           _PKG / "csrc" / "tri_score_tma.cuh", _PKG / "csrc" / "tri_calib.cuh",
+           _PKG / "csrc" / "tri_score_tma.cuh", _PKG / "csrc" / "tri_score_umma.cuh", _PKG / "csrc" / "tri_calib.cuh",
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",
-           "tri_compress", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_last_cuda_error",
+           "tri_compress", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_set_pipeline", "tri_set_score_kernel", "tri_last_cuda_error",
            "tri_profile_begin", "tri_profile_read", "tri_profile_end",
            "tri_calib_state_bytes", "tri_calib_workspace_bytes", "tri_calib_reset", "tri_calib_accumulate",
            "tri_calib_finalize", "tri_selftest_bounded_wait"]
@@ -105,7 +105,11 @@ def lib():
     L.tri_compress.restype = ctypes.c_int
     L.tri_compress_host.argtypes = [P, VP, VP, i32, P, P, i32, VP, VP, P, P, P, sz, P]
     L.tri_compress_host.restype = ctypes.c_int
-    L.tri_compress_launches.argtypes = [P, VP, VP]
+    L.tri_compress_launches.argtypes = [P, VP, i32, VP]
+    L.tri_set_pipeline.argtypes = [P, i32]
+    L.tri_set_pipeline.restype = ctypes.c_int
+    L.tri_set_score_kernel.argtypes = [P, i32]
+    L.tri_set_score_kernel.restype = ctypes.c_int
     L.tri_compress_launches.restype = i32
     for fn in (L.tri_profile_begin, L.tri_profile_end):
         fn.argtypes = [P]
@@ -322,9 +326,18 @@ class TriContext:
     def profile_end(self):
         _check(lib().tri_profile_end(self._h), "tri_profile_end")
 
-    def compress_launches(self, src: CacheView, dst: CacheView) -> int:
+    def compress_launches(self, src: CacheView, S: int, dst: CacheView) -> int:
         a, b = src.c_view(), dst.c_view()
-        return int(lib().tri_compress_launches(self._h, ctypes.byref(a), ctypes.byref(b)))
+        return int(lib().tri_compress_launches(self._h, ctypes.byref(a), S, ctypes.byref(b)))
+
+    def set_score_kernel(self, which: int):
+        """0: tcgen05 scoring kernel (default); 1: mma.sync scoring kernel.  Call before workspace()."""
+        _check(lib().tri_set_score_kernel(self._h, which), "tri_set_score_kernel")
+
+    def set_pipeline(self, ranges: int):
+        """0: ranges chosen per call (default); 1: the whole round on the caller's stream; n: n unit ranges with
+        selection and compaction on the context's side stream."""
+        _check(lib().tri_set_pipeline(self._h, ranges), "tri_set_pipeline")
 
 
 class Calibrator:

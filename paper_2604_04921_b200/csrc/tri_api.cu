@@ -14,12 +14,17 @@
 #include "tri_compact.cuh"
 #include "tri_score.cuh"
 #include "tri_score_tma.cuh"
+#include "tri_score_umma.cuh"
 #include "tri_select.cuh"
 
 using namespace tri;
 
 constexpr int kHostSlabs = 8;     // layer ranges tri_compress_host is pipelined over
-constexpr int kProfEvents = 6;   // boundaries of the 5 launches of tri_compress
+constexpr int kMaxRanges = 16;    // unit ranges one tri_compress may be issued over
+constexpr int kKinds = 5;         // kernel kinds timed while profiling: fold, score, normalise, select, compact
+constexpr int kMaxProf = 2 + 5 * kMaxRanges;   // launches of one round
+
+struct ProfRec { cudaEvent_t b, e; int kind; };
 
 struct tri_ctx {
     tri_model_desc desc;
@@ -28,19 +33,36 @@ struct tri_ctx {
     double2 *dbar_d;     // [64]  (1/|D|) sum_delta e^{i omega_f delta}
     float *qc_d;         // [L][H*G][128]
     float *mw_d;         // [L][H*G][64]   weight of |k_f| in the norm term
-    bool profiling;      // tri_profile_begin .. tri_profile_end: time each kernel of tri_compress
-    cudaEvent_t ev[kProfEvents];
+    // tri_profile_begin .. tri_profile_end: an event pair around every launch of tri_compress
+    bool profiling;
+    ProfRec prof[kMaxProf];
+    int prof_used;
     // tri_compress_host: device-to-host copies of one layer range run on `back` while the caller's stream
     // already brings in and compresses the next range
     cudaStream_t back;
     cudaEvent_t slab_done[kHostSlabs], back_done;
     bool have_back;
+    // tri_compress over unit ranges: selection and compaction of range i run on `side` (highest priority)
+    // while the caller's stream already scores range i + 1
+    cudaStream_t side;
+    cudaEvent_t scored[kMaxRanges], side_done;
+    bool have_side;
+    int pipeline;        // 0: number of ranges chosen per call, 1: single stream, n: n ranges
+    int score_kernel;    // bf16 keys: 0 = tcgen05 kernel (128-key tiles), 1 = mma.sync kernel (16-key warp tiles)
 };
 
-// Records event i on the stream while profiling is on (between the launches of tri_compress).
-static void mark(tri_ctx *c, int i, cudaStream_t st)
+// While profiling: an event before and after a launch, on the stream it goes to.  Returns the record's slot.
+static int prof_open(tri_ctx *c, int kind, cudaStream_t st)
 {
-    if (c->profiling) cudaEventRecord(c->ev[i], st);
+    if (!c->profiling || c->prof_used >= kMaxProf) return -1;
+    const int i = c->prof_used++;
+    c->prof[i].kind = kind;
+    cudaEventRecord(c->prof[i].b, st);
+    return i;
+}
+static void prof_close(tri_ctx *c, int i, cudaStream_t st)
+{
+    if (i >= 0) cudaEventRecord(c->prof[i].e, st);
 }
 
 // Named range on the calling host thread for timeline tools (a no-op when no tool is attached).
@@ -91,7 +113,11 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
     c->desc.offsets = nullptr;
     c->omega_d = nullptr; c->dbar_d = nullptr; c->qc_d = nullptr; c->mw_d = nullptr;
     c->profiling = false;
+    c->prof_used = 0;
     c->have_back = false;
+    c->have_side = false;
+    c->pipeline = 0;
+    c->score_kernel = 0;
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaGetDevice"); }
 
@@ -142,6 +168,21 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
             break;
         }
         c->have_back = true;
+        // the side stream of the pipelined round; without it (creation failed) rounds run on one stream
+        int least = 0, greatest = 0;
+        if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) { cudaGetLastError(); break; }
+        if (cudaStreamCreateWithPriority(&c->side, cudaStreamNonBlocking, greatest) != cudaSuccess) { cudaGetLastError(); break; }
+        int ok = 0;
+        for (; ok <= kMaxRanges; ++ok)
+            if (cudaEventCreateWithFlags(ok < kMaxRanges ? &c->scored[ok] : &c->side_done, cudaEventDisableTiming) != cudaSuccess)
+                break;
+        if (ok <= kMaxRanges) {
+            cudaGetLastError();
+            for (int i = 0; i < ok; ++i) cudaEventDestroy(c->scored[i]);
+            cudaStreamDestroy(c->side);
+            break;
+        }
+        c->have_side = true;
     } while (0);
     if (e != cudaSuccess) {
         st = cuda_fail(e, "tri_create");
@@ -155,7 +196,12 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
 extern "C" tri_status tri_destroy(tri_ctx *c)
 {
     if (!c) return TRI_OK;
-    if (c->profiling) for (int i = 0; i < kProfEvents; ++i) cudaEventDestroy(c->ev[i]);
+    if (c->profiling) tri_profile_end(c);
+    if (c->have_side) {
+        for (int i = 0; i < kMaxRanges; ++i) cudaEventDestroy(c->scored[i]);
+        cudaEventDestroy(c->side_done);
+        cudaStreamDestroy(c->side);
+    }
     if (c->have_back) {
         for (int i = 0; i < kHostSlabs; ++i) cudaEventDestroy(c->slab_done[i]);
         cudaEventDestroy(c->back_done);
@@ -181,14 +227,16 @@ struct Plan {
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-// Keys per scoring block: about 96 warp tiles (1,536 keys), evened out over the unit.
-void pick_chunk(int32_t n_max, int32_t *chunk, int32_t *nchunks)
+// Keys per scoring block, evened out over the unit: about 96 warp tiles of 16 keys (1,536 keys) for the mma.sync
+// kernel, about 16 tiles of 128 keys (2,048 keys) for the tcgen05 kernel.
+void pick_chunk(int32_t n_max, int score_kernel, int32_t *chunk, int32_t *nchunks)
 {
-    int32_t tiles = (n_max + kTileKeys - 1) / kTileKeys;
-    int32_t nch = (tiles + 48) / 96;
+    const int32_t tile = score_kernel == 0 ? kUTile : kTileKeys, want = score_kernel == 0 ? 16 : 96;
+    int32_t tiles = (n_max + tile - 1) / tile;
+    int32_t nch = (tiles + want / 2) / want;
     if (nch < 1) nch = 1;
     int32_t per = (tiles + nch - 1) / nch;
-    *chunk = per * kTileKeys;
+    *chunk = per * tile;
     *nchunks = (tiles + per - 1) / per;
 }
 
@@ -200,7 +248,7 @@ Plan make_plan(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget, int32
     Plan p;
     const int G = c->desc.group_size;
     p.U = (n_layers > 0 ? n_layers : c->desc.n_layers) * S * c->desc.n_kv_heads;
-    pick_chunk(n_max, &p.chunk, &p.nchunks);
+    pick_chunk(n_max, c->score_kernel, &p.chunk, &p.nchunks);
     size_t o = 0;
     p.off_E = o;      o += align256((size_t)S * kBands * sizeof(double2));
     p.off_raw = o;    o += align256((size_t)p.U * n_max * G * sizeof(float));
@@ -310,6 +358,12 @@ cudaError_t allow_score_smem()
     return cudaFuncSetAttribute(k_score_tma<NT, LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScoreDynSmem);
 }
 
+template <int NCOL, int LAYOUT>
+cudaError_t allow_umma_smem()
+{
+    return cudaFuncSetAttribute(k_score_umma<NCOL, LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, umma_smem_bytes(NCOL));
+}
+
 cudaError_t prepare_device()
 {
     cudaError_t e;
@@ -318,7 +372,11 @@ cudaError_t prepare_device()
     if ((e = allow_score_smem<4, 0>()) != cudaSuccess) return e;
     if ((e = allow_score_smem<1, 1>()) != cudaSuccess) return e;
     if ((e = allow_score_smem<2, 1>()) != cudaSuccess) return e;
-    return allow_score_smem<4, 1>();
+    if ((e = allow_score_smem<4, 1>()) != cudaSuccess) return e;
+    if ((e = allow_umma_smem<16, 0>()) != cudaSuccess) return e;
+    if ((e = allow_umma_smem<32, 0>()) != cudaSuccess) return e;
+    if ((e = allow_umma_smem<16, 1>()) != cudaSuccess) return e;
+    return allow_umma_smem<32, 1>();
 }
 
 // Every entry point that launches kernels runs on the device the context was created on.
@@ -348,11 +406,29 @@ tri_status launch_score_tma(int NT, dim3 grid, cudaStream_t st, const CUtensorMa
     return launch_score_tma_one<4, LAYOUT>(grid, st, map, sp);
 }
 
-// fold -> raw scores -> z-score/max (3 launches); without the last one when `scores` is NULL: the fused round
-// leaves the normalisation to its selection kernel.
+template <int LAYOUT>
+void launch_score_umma(int G, dim3 grid, cudaStream_t st, const CUtensorMap &map, const ScoreParams &sp)
+{
+    if (G <= 8) k_score_umma<16, LAYOUT><<<grid, kUThreads, umma_smem_bytes(16), st>>>(map, sp);
+    else k_score_umma<32, LAYOUT><<<grid, kUThreads, umma_smem_bytes(32), st>>>(map, sp);
+}
+
+// A contiguous range of units (u = (layer * S + seq) * H + head) one launch covers.
+struct Units { int32_t first, count; };
+
+tri_status run_fold(tri_ctx *c, int32_t S, const int64_t *cur_pos, char *ws, const Plan &pl, cudaStream_t st)
+{
+    const int pr = prof_open(c, 0, st);
+    k_fold_phasors<<<S, kBands, 0, st>>>(c->omega_d, c->dbar_d, cur_pos, (double2 *)(ws + pl.off_E));
+    prof_close(c, pr, st);
+    return check_launch("k_fold_phasors");
+}
+
+// raw scores -> z-score/max (2 launches) of the units `un`; without the last one when `scores` is NULL: the fused
+// round leaves the normalisation to its selection kernel.  The phasors must have been folded (run_fold).
 tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, float *scores,
                      float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st,
-                     Layers ly = Layers{0, 0}, int32_t skip_upto = 0)
+                     Units un, Layers ly = Layers{0, 0}, int32_t skip_upto = 0)
 {
     if (ly.count == 0) ly.count = c->desc.n_layers;
     const size_t head0 = (size_t)ly.first * c->desc.n_kv_heads * c->desc.group_size;   // first query head of the range
@@ -360,60 +436,61 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     double2 *E = (double2 *)(ws + pl.off_E);
     float *raw = raw_out ? raw_out : (float *)(ws + pl.off_raw);
     double2 *part = (double2 *)(ws + pl.off_part);
-
-    mark(c, 0, st);
-    k_fold_phasors<<<S, kBands, 0, st>>>(c->omega_d, c->dbar_d, cur_pos, E);
-    tri_status r = check_launch("k_fold_phasors");
-    if (r != TRI_OK) return r;
-    mark(c, 1, st);
+    tri_status r;
 
     ScoreParams sp;
     sp.src = to_view(src);
-    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G; sp.skip_upto = skip_upto;
+    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G; sp.u0 = un.first; sp.skip_upto = skip_upto;
     sp.chunk = pl.chunk; sp.nchunks = pl.nchunks;
     sp.E = E; sp.qc = c->qc_d + head0 * kHeadDim; sp.mw = c->mw_d + head0 * kBands;
     sp.raw = raw; sp.partials = part; sp.device_status = device_status;
-    dim3 grid((unsigned)((size_t)pl.U * pl.nchunks));
+    dim3 grid((unsigned)((size_t)un.count * pl.nchunks));
+    int pr = prof_open(c, 1, st);
     if (src->k_kind == 0) {
         int NT = G <= 4 ? 1 : (G <= 8 ? 2 : 4);
         CUtensorMap map;
         if ((r = encode_key_map(c, src, S, ly.count, &map)) != TRI_OK) return r;
-        r = c->desc.pair_layout == 0 ? launch_score_tma<0>(NT, grid, st, map, sp)
-                                     : launch_score_tma<1>(NT, grid, st, map, sp);
-        if (r != TRI_OK) return r;
+        if (c->score_kernel == 0) {
+            if (c->desc.pair_layout == 0) launch_score_umma<0>(G, grid, st, map, sp);
+            else launch_score_umma<1>(G, grid, st, map, sp);
+        } else {
+            r = c->desc.pair_layout == 0 ? launch_score_tma<0>(NT, grid, st, map, sp)
+                                         : launch_score_tma<1>(NT, grid, st, map, sp);
+            if (r != TRI_OK) return r;
+        }
     } else {
         if (c->desc.pair_layout == 0)
             k_score_f32_pre<0><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);
         else
             k_score_f32_pre<1><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);
     }
+    prof_close(c, pr, st);
     if ((r = check_launch("k_score")) != TRI_OK) return r;
-    mark(c, 2, st);
-    if (!scores) {
-        mark(c, 3, st);
-        return TRI_OK;
-    }
+    if (!scores) return TRI_OK;
 
     NormParams np;
     np.raw = raw; np.partials = part; np.seq_lens = src->seq_lens; np.scores = scores;
     np.S = S; np.H = c->desc.n_kv_heads; np.G = G; np.n_max = src->n_max;
-    np.chunk = pl.chunk; np.nchunks = pl.nchunks;
+    np.chunk = pl.chunk; np.nchunks = pl.nchunks; np.u0 = un.first;
+    pr = prof_open(c, 2, st);
     k_normalize<<<grid, 256, 0, st>>>(np);
-    r = check_launch("k_normalize");
-    mark(c, 3, st);
-    return r;
+    prof_close(c, pr, st);
+    return check_launch("k_normalize");
 }
 
-// Top-B selection.  pl == NULL: from the final scores in `scores` (tri_select).  pl != NULL: the fused round,
-// straight from the raw scores and partial sums in the workspace `ws`; final scores are parked in its score area.
+// Top-B selection of the units `un`.  pl == NULL: from the final scores in `scores` (tri_select).  pl != NULL: the
+// fused round, straight from the raw scores and partial sums in the workspace `ws`; final scores are parked in its
+// score area.
 tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
                       int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
-                      int32_t U, const Plan *pl, char *ws, cudaStream_t st)
+                      Units un, const Plan *pl, char *ws, cudaStream_t st)
 {
     SelectParams p;
     p.scores = scores; p.scores_w = nullptr; p.seq_lens = seq_lens; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
-    p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget;
+    p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget; p.u0 = un.first;
     p.raw = nullptr; p.partials = nullptr; p.G = c->desc.group_size; p.chunk = 0; p.nchunks = 0;
+    const int U = un.count;
+    const int pr = prof_open(c, 3, st);
     if (pl) {
         p.scores_w = (float *)(ws + pl->off_scores);
         p.scores = p.scores_w;
@@ -426,9 +503,8 @@ tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, 
         if (n_max <= kSelSmallUnit) k_select<false, 256><<<U, 256, 0, st>>>(p);
         else k_select<false, 1024><<<U, 1024, 0, st>>>(p);
     }
-    tri_status r = check_launch("k_select");
-    mark(c, 4, st);
-    return r;
+    prof_close(c, pr, st);
+    return check_launch("k_select");
 }
 
 bool aliases(const tri_cache_view *a, const tri_cache_view *b)
@@ -436,20 +512,28 @@ bool aliases(const tri_cache_view *a, const tri_cache_view *b)
     return a->k == b->k || (a->v && a->v == b->v) || (a->positions && a->positions == b->positions);
 }
 
+// Whether the round compacts bf16 K + V in place: then the gather is two launches (tiled prefix, parallel pass).
+bool two_pass_compaction(const tri_cache_view *src, const tri_cache_view *dst)
+{
+    return aliases(src, dst) && src->k_kind == 0 && src->v && dst->v;
+}
+
 tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx, const int32_t *kept_cnt,
                        int32_t S, int32_t budget, const tri_cache_view *dst, int32_t *new_seq_lens,
-                       int32_t *device_status, int32_t U, cudaStream_t st)
+                       int32_t *device_status, Units un, cudaStream_t st)
 {
     CompactParams p;
     p.src = to_view(src); p.dst = to_view(dst);
     p.kept_idx = kept_idx; p.kept_cnt = kept_cnt; p.new_seq_lens = new_seq_lens;
-    p.S = S; p.H = c->desc.n_kv_heads; p.budget = budget;
+    p.S = S; p.H = c->desc.n_kv_heads; p.budget = budget; p.u0 = un.first;
     p.k_esize = src->k_kind == 0 ? 2 : 4;
     p.k_vec = kHeadDim * p.k_esize / 16;
     p.v_vec = (src->v && dst->v) ? kHeadDim * 2 / 16 : 0;
     p.device_status = device_status;
     const bool rows16 = src->k_kind == 0 && p.v_vec != 0;     // bf16 K and V: the row-gather kernel applies
+    const int U = un.count;
     dim3 grid(U, (budget + kFastRowsPerBlock - 1) / kFastRowsPerBlock);
+    const int pr = prof_open(c, 4, st);
     if (aliases(src, dst)) {
         // in place: the prefix whose sources lie inside the destination range goes tile by tile in one block
         // per unit; everything behind it is a hazard-free gather
@@ -465,9 +549,22 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
         dim3 grid_any(U, (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock);
         k_gather_any<<<grid_any, kGatherThreads, 0, st>>>(p);
     }
-    tri_status r = check_launch("k_compact");
-    mark(c, 5, st);
-    return r;
+    prof_close(c, pr, st);
+    return check_launch("k_compact");
+}
+
+// Number of unit ranges a round over U units is issued in.  One range = everything on the caller's stream.
+// With several, selection and compaction of a range run on the context's side stream under the scoring of the
+// next: the latency-bound selection then costs HBM nothing.  Ranges stay wide (at least 32 units) so that every
+// launch still fills the GPU.
+int pick_ranges(const tri_ctx *c, int32_t U)
+{
+    if (!c->have_side) return 1;
+    int m = c->pipeline > 0 ? c->pipeline : U / 32;
+    if (c->pipeline == 0 && m > 8) m = 8;
+    if (m > kMaxRanges) m = kMaxRanges;
+    if (m > U) m = U;
+    return m < 1 ? 1 : m;
 }
 
 tri_status check_common(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget)
@@ -500,7 +597,8 @@ extern "C" tri_status tri_score(tri_ctx *c, const tri_cache_view *src, int32_t S
     if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
     Plan pl = make_plan(c, S, src->n_max, 0);
     if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
-    return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream);
+    if ((r = run_fold(c, S, cur_pos, (char *)ws, pl, (cudaStream_t)stream)) != TRI_OK) return r;
+    return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream, Units{0, pl.U});
 }
 
 extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S,
@@ -513,7 +611,7 @@ extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t 
     if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_common(c, S, n_max, budget)) != TRI_OK) return r;
     int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
-    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, U, nullptr, nullptr,
+    return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, Units{0, U}, nullptr, nullptr,
                       (cudaStream_t)stream);
 }
 
@@ -530,14 +628,15 @@ extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const i
     if (dst->n_max < budget && dst->n_max < src->n_max) return TRI_ERR_INVALID_ARG;
     if (src->k_kind != dst->k_kind) return TRI_ERR_INVALID_ARG;
     int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
-    return run_compact(c, src, kept_idx, kept_cnt, S, budget, dst, new_seq_lens, nullptr, U, (cudaStream_t)stream);
+    return run_compact(c, src, kept_idx, kept_cnt, S, budget, dst, new_seq_lens, nullptr, Units{0, U}, (cudaStream_t)stream);
 }
 
-// The fused round over a range of layers; the views start at the range's first layer.
+// The fused round over a range of layers; the views start at the range's first layer.  `ranges` > 1 issues it
+// over that many unit ranges, selection and compaction of each on the side stream.
 static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                                   int32_t budget, const tri_cache_view *dst, int32_t *kept_idx, int32_t *kept_cnt,
                                   int32_t *new_seq_lens, int32_t *device_status, void *ws, size_t ws_bytes,
-                                  cudaStream_t st)
+                                  cudaStream_t st, int ranges)
 {
     tri_status r;
     NvtxRange whole("tri_compress");
@@ -546,21 +645,47 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
     char *w = (char *)ws;
     int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
     int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
-    {
-        NvtxRange part("tri_compress: fold + score");
-        // sequences that do not exceed the budget are kept whole: their keys are not even read
-        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, ly, budget)) != TRI_OK) return r;
-    }
-    {
-        NvtxRange part("tri_compress: normalise + select");
+    c->prof_used = 0;
+    if ((r = run_fold(c, S, cur_pos, w, pl, st)) != TRI_OK) return r;
+    if (ranges <= 1) {
+        const Units all{0, pl.U};
+        {
+            NvtxRange part("tri_compress: score");
+            // sequences that do not exceed the budget are kept whole: their keys are not even read
+            if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, all, ly, budget)) != TRI_OK) return r;
+        }
+        {
+            NvtxRange part("tri_compress: normalise + select");
+            if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, all, &pl, w, st)) != TRI_OK)
+                return r;
+        }
         // new_seq_lens may be the very array the scoring and selection kernels read the lengths from, so only the
         // last launch of the round (the gather, which reads kept counts, never lengths) stores it
-        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, pl.U, &pl, w,
-                            st)) != TRI_OK)
-            return r;
+        NvtxRange part("tri_compress: compact");
+        return run_compact(c, src, idx, cnt, S, budget, dst, new_seq_lens, device_status, all, st);
     }
-    NvtxRange part("tri_compress: compact");
-    return run_compact(c, src, idx, cnt, S, budget, dst, new_seq_lens, device_status, pl.U, st);
+    // Pipelined: the caller's stream scores range after range; behind each range an event lets the side stream
+    // select and compact it while the next range is being scored.  The caller's stream waits for the side stream
+    // at the end, so the round is complete for whatever the caller enqueues next (and for a graph capture the
+    // side stream has joined again).
+    for (int i = 0; i < ranges; ++i) {
+        const int32_t a = (int32_t)((int64_t)pl.U * i / ranges), b = (int32_t)((int64_t)pl.U * (i + 1) / ranges);
+        const Units un{a, b - a};
+        if (un.count == 0) continue;
+        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, un, ly, budget)) != TRI_OK) return r;
+        TRI_CUDA(cudaEventRecord(c->scored[i], st));
+        TRI_CUDA(cudaStreamWaitEvent(c->side, c->scored[i], 0));
+        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, un, &pl, w, c->side)) != TRI_OK) return r;
+        if ((r = run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, un, c->side)) != TRI_OK) return r;
+    }
+    TRI_CUDA(cudaEventRecord(c->side_done, c->side));
+    TRI_CUDA(cudaStreamWaitEvent(st, c->side_done, 0));
+    if (new_seq_lens) {
+        // after every kernel that reads the lengths (new_seq_lens may be that very array)
+        k_store_lens<<<(S + 255) / 256, 256, 0, st>>>(src->seq_lens, new_seq_lens, S, src->n_max, budget);
+        return check_launch("k_store_lens");
+    }
+    return TRI_OK;
 }
 
 extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
@@ -577,17 +702,32 @@ extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_
     if (dst->n_max < budget && dst->n_max < src->n_max) return TRI_ERR_INVALID_ARG;
     if (src->k_kind != dst->k_kind) return TRI_ERR_INVALID_ARG;
     if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
+    const int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
     return compress_layers(c, Layers{0, c->desc.n_layers}, src, S, cur_pos, budget, dst, kept_idx, kept_cnt, new_seq_lens,
-                           device_status, ws, ws_bytes, (cudaStream_t)stream);
+                           device_status, ws, ws_bytes, (cudaStream_t)stream, pick_ranges(c, U));
 }
 
-extern "C" int32_t tri_compress_launches(const tri_ctx *c, const tri_cache_view *src, const tri_cache_view *dst)
+extern "C" tri_status tri_set_pipeline(tri_ctx *c, int32_t ranges)
 {
-    (void)c;
-    if (!src || !dst) return 0;
-    // fold, score, select (which also normalises), gather; an in-place round of bf16 K + V splits the gather into
-    // the tiled prefix pass and the parallel pass behind it
-    return 4 + ((aliases(src, dst) && src->k_kind == 0 && src->v && dst->v) ? 1 : 0);
+    if (!c || ranges < 0 || ranges > kMaxRanges) return TRI_ERR_INVALID_ARG;
+    c->pipeline = ranges;
+    return TRI_OK;
+}
+
+extern "C" tri_status tri_set_score_kernel(tri_ctx *c, int32_t which)
+{
+    if (!c || which < 0 || which > 1) return TRI_ERR_INVALID_ARG;
+    c->score_kernel = which;
+    return TRI_OK;
+}
+
+extern "C" int32_t tri_compress_launches(const tri_ctx *c, const tri_cache_view *src, int32_t S, const tri_cache_view *dst)
+{
+    if (!c || !src || !dst || S <= 0) return 0;
+    // the phasor fold, then per unit range: score, select (which also normalises), gather; an in-place round of
+    // bf16 K + V splits the gather into the tiled prefix pass and the parallel pass behind it
+    const int m = pick_ranges(c, c->desc.n_layers * S * c->desc.n_kv_heads);
+    return 1 + m * (3 + (two_pass_compaction(src, dst) ? 1 : 0));
 }
 
 extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_host, const tri_cache_view *src_dev,
@@ -667,7 +807,7 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
         if (dst_dev->v) dv.v = (char *)dst_dev->v + dof * 2;
         if (dst_dev->positions) dv.positions = dst_dev->positions + u0 * dst_dev->n_max;
         if ((r = compress_layers(c, Layers{l0, nl}, &sv, S, cur_pos_dev, budget, &dv, nullptr, kept_cnt_dev + u0, nullptr,
-                                 nullptr, ws, ws_bytes, st)) != TRI_OK)
+                                 nullptr, ws, ws_bytes, st, 1)) != TRI_OK)
             return r;
         if (M > 1) {
             TRI_CUDA(cudaEventRecord(c->slab_done[i], st));
@@ -703,13 +843,15 @@ extern "C" tri_status tri_profile_begin(tri_ctx *c)
 {
     if (!c) return TRI_ERR_INVALID_ARG;
     if (c->profiling) return TRI_OK;
-    for (int i = 0; i < kProfEvents; ++i) {
-        cudaError_t e = cudaEventCreate(&c->ev[i]);
+    for (int i = 0; i < kMaxProf; ++i) {
+        cudaError_t e = cudaEventCreate(&c->prof[i].b);
+        if (e == cudaSuccess && (e = cudaEventCreate(&c->prof[i].e)) != cudaSuccess) cudaEventDestroy(c->prof[i].b);
         if (e != cudaSuccess) {
-            for (int j = 0; j < i; ++j) cudaEventDestroy(c->ev[j]);
+            for (int j = 0; j < i; ++j) { cudaEventDestroy(c->prof[j].b); cudaEventDestroy(c->prof[j].e); }
             return cuda_fail(e, "cudaEventCreate");
         }
     }
+    c->prof_used = 0;
     c->profiling = true;
     return TRI_OK;
 }
@@ -717,16 +859,23 @@ extern "C" tri_status tri_profile_begin(tri_ctx *c)
 extern "C" tri_status tri_profile_read(tri_ctx *c, float *ms)
 {
     if (!c || !ms || !c->profiling) return TRI_ERR_INVALID_ARG;
-    TRI_CUDA(cudaEventSynchronize(c->ev[kProfEvents - 1]));
-    for (int i = 0; i + 1 < kProfEvents; ++i) TRI_CUDA(cudaEventElapsedTime(&ms[i], c->ev[i], c->ev[i + 1]));
+    for (int k = 0; k < kKinds; ++k) ms[k] = 0.f;
+    for (int i = 0; i < c->prof_used; ++i) {
+        float t = 0.f;
+        TRI_CUDA(cudaEventSynchronize(c->prof[i].e));
+        TRI_CUDA(cudaEventElapsedTime(&t, c->prof[i].b, c->prof[i].e));
+        ms[c->prof[i].kind] += t;
+    }
     return TRI_OK;
 }
 
 extern "C" tri_status tri_profile_end(tri_ctx *c)
 {
     if (!c) return TRI_ERR_INVALID_ARG;
-    if (c->profiling) for (int i = 0; i < kProfEvents; ++i) cudaEventDestroy(c->ev[i]);
+    if (c->profiling)
+        for (int i = 0; i < kMaxProf; ++i) { cudaEventDestroy(c->prof[i].b); cudaEventDestroy(c->prof[i].e); }
     c->profiling = false;
+    c->prof_used = 0;
     return TRI_OK;
 }
 
@@ -775,7 +924,8 @@ extern "C" tri_status tri_score_static(tri_ctx *c, const tri_cache_view *src, in
     if (dev != c->device || dev < 0 || dev >= kMaxDevices) return TRI_ERR_INVALID_ARG;
     void *ws = nullptr;
     if ((r = score_scratch_address(dev, &ws)) != TRI_OK) return r;
-    return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream);
+    if ((r = run_fold(c, S, cur_pos, (char *)ws, pl, (cudaStream_t)stream)) != TRI_OK) return r;
+    return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream, Units{0, pl.U});
 }
 
 // ----------------------------------------------------------------------------------------------

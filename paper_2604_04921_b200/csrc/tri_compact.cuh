@@ -16,6 +16,7 @@ struct CompactParams {
     const int32_t *kept_cnt;   // [U]
     int32_t *new_seq_lens;     // [S] or NULL
     int32_t S, H, budget;
+    int32_t u0;                // first unit of this launch
     int32_t k_vec;             // 16-byte vectors per K row (16 for bf16, 32 for fp32)
     int32_t v_vec;             // 16-byte vectors per V row (16, or 0 without a value cache)
     int32_t k_esize;           // bytes per K element
@@ -67,7 +68,7 @@ constexpr int kInplaceRows = 128;       // rows per tile of the in-place schedul
 template <bool AFTER_PREFIX>
 __global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const CompactParams p)
 {
-    const int u = blockIdx.x;
+    const int u = p.u0 + blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
     if (!AFTER_PREFIX && blockIdx.y == 0 && threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0)
@@ -121,7 +122,7 @@ __global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const Compact
 // grid = (U, ceil(budget / 64)); a warp moves 8 rows at a time, 16 bytes per lane.
 __global__ void __launch_bounds__(kGatherThreads) k_gather_any(const CompactParams p)
 {
-    const int u = blockIdx.x;
+    const int u = p.u0 + blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
     if (blockIdx.y == 0 && threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0) p.new_seq_lens[s] = cnt;
@@ -194,7 +195,7 @@ static_assert(kInplaceRows == (kInplaceThreads / 32) * kFastRows, "a tile is 8 r
 
 __global__ void __launch_bounds__(kInplaceThreads, 2) k_compact_inplace_rows(const CompactParams p)
 {
-    const int u = blockIdx.x;
+    const int u = p.u0 + blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
     if (threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0) p.new_seq_lens[s] = cnt;
@@ -251,7 +252,7 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace_any(const C
 {
     __shared__ uint4 stage[kInplaceAnyRows * 48];
     __shared__ int32_t pos_s[kInplaceAnyRows];
-    const int u = blockIdx.x;
+    const int u = p.u0 + blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
     if (threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0) p.new_seq_lens[s] = cnt;
@@ -295,6 +296,14 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace_any(const C
             p.dst.positions[(int64_t)u * p.dst.n_max + j0 + threadIdx.x] = pos_s[threadIdx.x];
         __syncthreads();
     }
+}
+
+// new_seq_lens[s] = min(seq_lens[s], n_max, budget): the last launch of a round issued over several unit ranges (the two
+// arrays may be one and the same, and every earlier kernel reads the old lengths).
+__global__ void k_store_lens(const int32_t *seq_lens, int32_t *new_seq_lens, int32_t S, int32_t n_max, int32_t budget)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < S) new_seq_lens[s] = min(min(seq_lens[s], n_max), budget);
 }
 
 }  // namespace tri

@@ -91,6 +91,7 @@ __device__ __forceinline__ uint32_t bf16_hi_bits(float w)   // bf16(w), round to
 struct ScoreParams {
     View src;
     int32_t S, H, G;
+    int32_t u0;           // first unit of this launch (a round may be issued as several launches over unit ranges)
     int32_t skip_upto;    // units of at most this many keys are not scored (the fused round keeps them whole); 0 = score all
     int32_t chunk;        // keys per block (multiple of 16)
     int32_t nchunks;      // blocks per unit
@@ -114,7 +115,7 @@ k_score_f32_pre(const ScoreParams p, const double *__restrict__ omega, const dou
 {
     __shared__ double red[kScoreWarps][kMaxGroup][2];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int u = blockIdx.x / p.nchunks, chunk = blockIdx.x - u * p.nchunks;
+    const int ub = blockIdx.x / p.nchunks, chunk = blockIdx.x - ub * p.nchunks, u = p.u0 + ub;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int n = min(__ldg(p.src.seq_lens + s), p.src.n_max);
     const int key_begin = chunk * p.chunk;
@@ -233,14 +234,14 @@ struct NormParams {
     const double2 *partials;    // [U][nchunks][G]
     const int32_t *seq_lens;
     float *scores;              // [U][n_max]
-    int32_t S, H, G, n_max, chunk, nchunks;
+    int32_t S, H, G, n_max, chunk, nchunks, u0;
 };
 
 __global__ void __launch_bounds__(256) k_normalize(const NormParams p)
 {
     __shared__ float mu_s[kMaxGroup], rs_s[kMaxGroup];
     const int tid = threadIdx.x;
-    const int u = blockIdx.x / p.nchunks, chunk = blockIdx.x - u * p.nchunks;
+    const int ub = blockIdx.x / p.nchunks, chunk = blockIdx.x - ub * p.nchunks, u = p.u0 + ub;
     const int s = (u / p.H) % p.S;
     const int n = min(__ldg(p.seq_lens + s), p.n_max);
     const int key_begin = chunk * p.chunk;

@@ -107,7 +107,7 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
     __shared__ __align__(8) uint64_t bars[kScoreWarps][kStages];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int u = blockIdx.x / p.nchunks, chunk = blockIdx.x - u * p.nchunks;
+    const int ub = blockIdx.x / p.nchunks, chunk = blockIdx.x - ub * p.nchunks, u = p.u0 + ub;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int n = min(__ldg(p.src.seq_lens + s), p.src.n_max);
     const int key_begin = chunk * p.chunk;

@@ -34,6 +34,7 @@ struct SelectParams {
     int32_t *kept_idx;        // [U][budget]
     int32_t *kept_cnt;        // [U]
     int32_t S, H, n_max, budget;
+    int32_t u0;               // first unit of this launch
     // FUSED only: raw scores and partial sums of the scoring kernel
     const float *raw;         // [U][n_max][G]
     const double2 *partials;  // [U][nchunks][G]
@@ -111,7 +112,7 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
     __shared__ float mu_s[kMaxGroup], rs_s[kMaxGroup];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int u = blockIdx.x;
+    const int u = p.u0 + blockIdx.x;
     const int s = (u / p.H) % p.S;
     const int n = min(__ldg(p.seq_lens + s), p.n_max);
     const float *sc = p.scores + (int64_t)u * p.n_max;

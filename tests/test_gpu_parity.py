@@ -456,6 +456,36 @@ def test_host_resident_cache_round(pinned, budget):
         assert bool(torch.isnan(dv.float()).all()) and bool((dpos == -7).all())
 
 
+@pytest.mark.parametrize("kind", ["oneshot", "paged_in_place"])
+def test_pipelined_round_is_bit_identical(kind):
+    """tri_set_pipeline: the round issued over 1, 2, 5 and 16 unit ranges (selection and compaction on the context's
+    side stream under the scoring of the next range) gives the same bits as the single-stream round, and the
+    caller's stream sees the finished round."""
+    if kind == "oneshot":
+        sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="pipe", n_layers=3, n_kv_heads=3, n_keys=4000, budget=300)
+    else:
+        sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name="pipe_p", n_layers=3, n_kv_heads=2, n_seqs=3, n_keys=3000,
+                                                      n_keys_min=200, budget=512)
+    w = W.make_workload(sp, DEV)
+    k0, v0 = w.k.clone(), w.v.clone()
+    u = (2, sp.n_seqs - 1, 1)
+    oref = oracle_unit(w, *u, sp.budget)                     # before any in-place write
+    ctx = make_ctx(w)
+    ref = None
+    for ranges in (1, 2, 5, 16, 0):
+        w.k.copy_(k0); w.v.copy_(v0)
+        ctx.set_pipeline(ranges)
+        res = run_compress(w, sp.budget, ctx=ctx, in_place=(kind != "oneshot"), want_scores=False)
+        assert int(res["status"].item()) == 0
+        check_unit(w, res, oref, *u, sp.budget)
+        got = dict(idx=res["kept_idx"].clone(), cnt=res["kept_cnt"].clone(), lens=res["new_seq_lens"].clone(),
+                   k=res["k_out"].clone().view(torch.int16), v=res["v_out"].clone().view(torch.int16))
+        if ref is None:
+            ref = got
+        for key in ref:
+            assert torch.equal(ref[key], got[key]), (ranges, key)
+
+
 def test_round_replays_from_a_cuda_graph():
     """tri_compress only enqueues kernels on the given stream (no allocation, no synchronisation), so a decode
     loop can capture one round in a CUDA graph and replay it; the replay reads cur_pos from device memory."""
