@@ -222,16 +222,16 @@ namespace {
 
 struct Plan {
     int32_t U, chunk, nchunks;
-    size_t off_E, off_raw, off_part, off_scores, off_idx, off_cnt, total;
+    size_t off_E, off_bt, off_bn, off_raw, off_part, off_scores, off_idx, off_cnt, total;
 };
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 // Keys per scoring block, evened out over the unit: about 96 warp tiles of 16 keys (1,536 keys) for the mma.sync
-// kernel, about 16 tiles of 128 keys (2,048 keys) for the tcgen05 kernel.
+// kernel, about 32 tiles of 128 keys (4,096 keys) for the tcgen05 kernel.
 void pick_chunk(int32_t n_max, int score_kernel, int32_t *chunk, int32_t *nchunks)
 {
-    const int32_t tile = score_kernel == 0 ? kUTile : kTileKeys, want = score_kernel == 0 ? 16 : 96;
+    const int32_t tile = score_kernel == 0 ? kUTile : kTileKeys, want = score_kernel == 0 ? 32 : 96;
     int32_t tiles = (n_max + tile - 1) / tile;
     int32_t nch = (tiles + want / 2) / want;
     if (nch < 1) nch = 1;
@@ -251,6 +251,10 @@ Plan make_plan(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget, int32
     pick_chunk(n_max, c->score_kernel, &p.chunk, &p.nchunks);
     size_t o = 0;
     p.off_E = o;      o += align256((size_t)S * kBands * sizeof(double2));
+    // tcgen05 kernel: folded B operands per unit (trig) and per (layer, KV head) (norm), 256 bytes per accumulator column
+    const size_t ncol = c->score_kernel == 0 ? (G <= 8 ? 16 : 32) : 0;
+    p.off_bt = o;     o += align256((size_t)p.U * ncol * 256);
+    p.off_bn = o;     o += align256((size_t)(p.U / S) * ncol * 256);
     p.off_raw = o;    o += align256((size_t)p.U * n_max * G * sizeof(float));
     p.off_part = o;   o += align256((size_t)p.U * p.nchunks * G * sizeof(double2));
     p.off_scores = o; o += align256((size_t)p.U * n_max * sizeof(float));
@@ -416,12 +420,31 @@ void launch_score_umma(int G, dim3 grid, cudaStream_t st, const CUtensorMap &map
 // A contiguous range of units (u = (layer * S + seq) * H + head) one launch covers.
 struct Units { int32_t first, count; };
 
-tri_status run_fold(tri_ctx *c, int32_t S, const int64_t *cur_pos, char *ws, const Plan &pl, cudaStream_t st)
+template <int LAYOUT>
+void launch_fold_operands(int G, int U, cudaStream_t st, const OperandParams &op)
+{
+    if (G <= 8) k_fold_operands<16, LAYOUT><<<U, 256, 0, st>>>(op);
+    else k_fold_operands<32, LAYOUT><<<U, 512, 0, st>>>(op);
+}
+
+// Fold of everything the scoring kernels need that does not depend on the keys: the phasors of every sequence and,
+// for the tcgen05 kernel on bf16 keys, the B operands of its two contractions.
+tri_status run_fold(tri_ctx *c, int32_t S, const int64_t *cur_pos, char *ws, const Plan &pl, cudaStream_t st,
+                    bool bf16_keys = true, Layers ly = Layers{0, 0})
 {
     const int pr = prof_open(c, 0, st);
     k_fold_phasors<<<S, kBands, 0, st>>>(c->omega_d, c->dbar_d, cur_pos, (double2 *)(ws + pl.off_E));
+    if (c->score_kernel == 0 && bf16_keys) {
+        const size_t head0 = (size_t)ly.first * c->desc.n_kv_heads * c->desc.group_size;
+        OperandParams op;
+        op.E = (const double2 *)(ws + pl.off_E); op.qc = c->qc_d + head0 * kHeadDim; op.mw = c->mw_d + head0 * kBands;
+        op.bt = (uint8_t *)(ws + pl.off_bt); op.bn = (uint8_t *)(ws + pl.off_bn);
+        op.S = S; op.H = c->desc.n_kv_heads; op.G = c->desc.group_size;
+        if (c->desc.pair_layout == 0) launch_fold_operands<0>(op.G, pl.U, st, op);
+        else launch_fold_operands<1>(op.G, pl.U, st, op);
+    }
     prof_close(c, pr, st);
-    return check_launch("k_fold_phasors");
+    return check_launch("k_fold");
 }
 
 // raw scores -> z-score/max (2 launches) of the units `un`; without the last one when `scores` is NULL: the fused
@@ -443,6 +466,7 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G; sp.u0 = un.first; sp.skip_upto = skip_upto;
     sp.chunk = pl.chunk; sp.nchunks = pl.nchunks;
     sp.E = E; sp.qc = c->qc_d + head0 * kHeadDim; sp.mw = c->mw_d + head0 * kBands;
+    sp.bt = (const uint8_t *)(ws + pl.off_bt); sp.bn = (const uint8_t *)(ws + pl.off_bn);
     sp.raw = raw; sp.partials = part; sp.device_status = device_status;
     dim3 grid((unsigned)((size_t)un.count * pl.nchunks));
     int pr = prof_open(c, 1, st);
@@ -597,7 +621,7 @@ extern "C" tri_status tri_score(tri_ctx *c, const tri_cache_view *src, int32_t S
     if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
     Plan pl = make_plan(c, S, src->n_max, 0);
     if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
-    if ((r = run_fold(c, S, cur_pos, (char *)ws, pl, (cudaStream_t)stream)) != TRI_OK) return r;
+    if ((r = run_fold(c, S, cur_pos, (char *)ws, pl, (cudaStream_t)stream, src->k_kind == 0)) != TRI_OK) return r;
     return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream, Units{0, pl.U});
 }
 
@@ -646,7 +670,7 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
     int32_t *idx = kept_idx ? kept_idx : (int32_t *)(w + pl.off_idx);
     int32_t *cnt = kept_cnt ? kept_cnt : (int32_t *)(w + pl.off_cnt);
     c->prof_used = 0;
-    if ((r = run_fold(c, S, cur_pos, w, pl, st)) != TRI_OK) return r;
+    if ((r = run_fold(c, S, cur_pos, w, pl, st, src->k_kind == 0, ly)) != TRI_OK) return r;
     if (ranges <= 1) {
         const Units all{0, pl.U};
         {
@@ -924,7 +948,7 @@ extern "C" tri_status tri_score_static(tri_ctx *c, const tri_cache_view *src, in
     if (dev != c->device || dev < 0 || dev >= kMaxDevices) return TRI_ERR_INVALID_ARG;
     void *ws = nullptr;
     if ((r = score_scratch_address(dev, &ws)) != TRI_OK) return r;
-    if ((r = run_fold(c, S, cur_pos, (char *)ws, pl, (cudaStream_t)stream)) != TRI_OK) return r;
+    if ((r = run_fold(c, S, cur_pos, (char *)ws, pl, (cudaStream_t)stream, src->k_kind == 0)) != TRI_OK) return r;
     return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream, Units{0, pl.U});
 }
 

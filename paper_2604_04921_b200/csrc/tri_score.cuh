@@ -98,6 +98,8 @@ struct ScoreParams {
     const double2 *E;     // [S][64]  e^{i omega_f p_q} Dbar_f
     const float *qc;      // [L][H*G][128]  E[q_f]
     const float *mw;      // [L][H*G][64]   norm weights m_f
+    const uint8_t *bt;    // tcgen05 kernel: folded B operand images, [U] trig and [L*H] norm (see k_fold_operands)
+    const uint8_t *bn;
     float *raw;           // [U][n_max][G]
     double2 *partials;    // [U][nchunks][G]  (sum, sum of squares) of raw over the block's keys
     int32_t *device_status;
