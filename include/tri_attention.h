@@ -213,22 +213,24 @@ tri_status tri_score_static(tri_ctx *ctx, const tri_cache_view *src, int32_t S, 
 
 /*
  * How tri_compress is issued (the paper has no counterpart; a scheduling choice of this library).
- *   ranges = 1   every kernel of the round on the caller's stream, one launch each.
+ *   ranges = 1   (default) every kernel of the round on the caller's stream, one launch each.
  *   ranges > 1   the units are cut into that many contiguous ranges (at most 16).  The caller's stream scores range
  *                after range; selection and compaction of a range run on a high-priority stream owned by the context
  *                while the next range is being scored, so the latency-bound selection overlaps the key stream.  The
  *                caller's stream waits for that stream before tri_compress returns control to it: work enqueued on
  *                `stream` afterwards sees the finished round, and a stream capture sees the side stream joined.
- *   ranges = 0   (default) chosen per call: about one range per 32 units, at most 8.
+ *   ranges = 0   chosen per call: about one range per 32 units, at most 8.
  * Results are bit-identical in every mode.  One context must not run two tri_compress calls concurrently.
+ * On B200 the single-stream order measured fastest on every benchmark shape (the selection blocks take shared
+ * memory and thread slots from the scoring blocks they overlap), which is why it is the default.
  */
 tri_status tri_set_pipeline(tri_ctx *ctx, int32_t ranges);
 
 /*
  * Which kernel scores bf16 keys (the paper has no counterpart; both compute the same Sections 4.1-4.2 scores to
  * fp32 rounding, so results may differ in the last bits between the two, never within one):
- *   0 (default)  tcgen05: 128-key tiles, tensor-memory accumulator, magnitudes staged through shared memory
- *   1            mma.sync: 16-key warp tiles, everything in registers
+ *   0   tcgen05: 128-key tiles, accumulator and magnitude operand in tensor memory (default for group_size > 4)
+ *   1   mma.sync: 16-key warp tiles, everything in registers (default for group_size <= 4)
  * Call it before tri_workspace_bytes: the workspace layout depends on the kernel's block size.
  */
 tri_status tri_set_score_kernel(tri_ctx *ctx, int32_t which);

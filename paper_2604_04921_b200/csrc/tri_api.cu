@@ -116,8 +116,10 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
     c->prof_used = 0;
     c->have_back = false;
     c->have_side = false;
-    c->pipeline = 0;
-    c->score_kernel = 0;
+    c->pipeline = 1;
+    // Measured on B200: at G <= 4 the mma.sync kernel already streams at the copy rate and draws less power; from
+    // G = 5 on its tensor and issue load grows with G while the tcgen05 kernel's does not (5.8 against 5.5 TB/s at G = 8).
+    c->score_kernel = desc->group_size > 4 ? 0 : 1;
     cudaError_t e = cudaGetDevice(&c->device);
     if (e != cudaSuccess) { delete c; return cuda_fail(e, "cudaGetDevice"); }
 
@@ -577,10 +579,9 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
     return check_launch("k_compact");
 }
 
-// Number of unit ranges a round over U units is issued in.  One range = everything on the caller's stream.
-// With several, selection and compaction of a range run on the context's side stream under the scoring of the
-// next: the latency-bound selection then costs HBM nothing.  Ranges stay wide (at least 32 units) so that every
-// launch still fills the GPU.
+// Number of unit ranges a round over U units is issued in.  One range = everything on the caller's stream (the
+// default).  With several, selection and compaction of a range run on the context's side stream under the scoring of
+// the next.  0 asks for an automatic count: about one range per 32 units, at most 8.
 int pick_ranges(const tri_ctx *c, int32_t U)
 {
     if (!c->have_side) return 1;
