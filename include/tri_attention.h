@@ -162,6 +162,40 @@ tri_status tri_compress(tri_ctx *ctx, const tri_cache_view *src, int32_t S, cons
                         void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Head-specific budgets (Appendix A lists them as future work; the paper gives no allocation rule, so the budgets
+ * are the caller's).  The same calls with one budget per unit:
+ *   unit_budgets   device [U] int32; unit u keeps min(unit_budgets[u], budget, seq_lens[s]) rows (negative = 0)
+ *   budget         now only the capacity: row stride of kept_idx and upper bound of every unit's budget
+ * kept_cnt [U] is the per-unit row count afterwards.  A cache view carries one length per sequence, so new_seq_lens[s]
+ * receives the largest count among the sequence's units; rows between a unit's own count and that length are stale,
+ * and a later round over such a cache has to be issued per group of units with equal length.
+ */
+tri_status tri_select_budgets(tri_ctx *ctx, const float *scores, const int32_t *seq_lens, int32_t S,
+                              int32_t n_max, int32_t budget, const int32_t *unit_budgets, int32_t *kept_idx,
+                              int32_t *kept_cnt, void *stream);
+tri_status tri_compress_budgets(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                int32_t budget, const int32_t *unit_budgets, const tri_cache_view *dst,
+                                int32_t *kept_idx, int32_t *kept_cnt, int32_t *new_seq_lens,
+                                int32_t *device_status, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The round behind its window trigger (Section 4.3: pruning runs once per window of beta = 128 decoded tokens, and only on
+ * a cache that exceeds its budget), decided on the device so that a decode loop -- or a captured CUDA graph -- can issue
+ * this call after every step and have it do nothing until a sequence is due.
+ *   decoded   device [S] int32, owned by the caller, zero at the start of a sequence: tokens decoded since the
+ *             sequence's last window boundary.  The call adds `step` (tokens appended since the previous call); where
+ *             the sum reaches `beta` the count starts over and the sequence is due if seq_lens[s] > budget.
+ * Due sequences are compressed exactly as by tri_compress.  For the others no key is read and no row moves; their
+ * kept_cnt entries are 0, their kept_idx entries untouched and new_seq_lens[s] = seq_lens[s] (the two may be one array).
+ * Everything else as in tri_compress; a call in which nothing is due costs the round's launches, whose blocks exit at once.
+ */
+tri_status tri_compress_windowed(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                 int32_t budget, int32_t *decoded, int32_t step, int32_t beta,
+                                 const tri_cache_view *dst, int32_t *kept_idx, int32_t *kept_cnt,
+                                 int32_t *new_seq_lens, int32_t *device_status, void *ws, size_t ws_bytes,
+                                 void *stream);
+
+/*
  * The fused round for a cache that lives in HOST memory (contiguous views only): copies K of src to the
  * device staging view, runs tri_compress, and copies the compacted rows, positions and counts back, all
  * on `stream`.  V and positions are needed only for the kept rows: if at most half of the rows can be kept

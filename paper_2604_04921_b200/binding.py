@@ -24,7 +24,7 @@ HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cu
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",
-           "tri_compress", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_set_pipeline", "tri_set_score_kernel", "tri_last_cuda_error",
+           "tri_compress", "tri_select_budgets", "tri_compress_budgets", "tri_compress_windowed", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_set_pipeline", "tri_set_score_kernel", "tri_last_cuda_error",
            "tri_profile_begin", "tri_profile_read", "tri_profile_end",
            "tri_calib_state_bytes", "tri_calib_workspace_bytes", "tri_calib_reset", "tri_calib_accumulate",
            "tri_calib_finalize", "tri_selftest_bounded_wait"]
@@ -103,6 +103,12 @@ def lib():
     L.tri_compact.restype = ctypes.c_int
     L.tri_compress.argtypes = [P, VP, i32, P, i32, VP, P, P, P, P, P, sz, P]
     L.tri_compress.restype = ctypes.c_int
+    L.tri_select_budgets.argtypes = [P, P, P, i32, i32, i32, P, P, P, P]
+    L.tri_select_budgets.restype = ctypes.c_int
+    L.tri_compress_budgets.argtypes = [P, VP, i32, P, i32, P, VP, P, P, P, P, P, sz, P]
+    L.tri_compress_budgets.restype = ctypes.c_int
+    L.tri_compress_windowed.argtypes = [P, VP, i32, P, i32, P, i32, i32, VP, P, P, P, P, P, sz, P]
+    L.tri_compress_windowed.restype = ctypes.c_int
     L.tri_compress_host.argtypes = [P, VP, VP, i32, P, P, i32, VP, VP, P, P, P, sz, P]
     L.tri_compress_host.restype = ctypes.c_int
     L.tri_compress_launches.argtypes = [P, VP, i32, VP]
@@ -272,11 +278,17 @@ class TriContext:
         _check(code, "tri_score_static")
 
     def select(self, scores: torch.Tensor, seq_lens: torch.Tensor, n_max: int, budget: int,
-               kept_idx: torch.Tensor, kept_cnt: torch.Tensor, ws: Optional[torch.Tensor] = None):
+               kept_idx: torch.Tensor, kept_cnt: torch.Tensor, ws: Optional[torch.Tensor] = None,
+               unit_budgets: Optional[torch.Tensor] = None):
         S = seq_lens.shape[0]
         assert scores.dtype == torch.float32 and scores.is_contiguous() and scores.numel() == self.units(S) * n_max
         assert kept_idx.dtype == torch.int32 and kept_idx.numel() == self.units(S) * budget
         assert kept_cnt.dtype == torch.int32 and kept_cnt.numel() == self.units(S)
+        if unit_budgets is not None:
+            assert unit_budgets.dtype == torch.int32 and unit_budgets.numel() == self.units(S) and unit_budgets.is_contiguous()
+            _check(lib().tri_select_budgets(self._h, _ptr(scores), _ptr(seq_lens), S, n_max, budget, _ptr(unit_budgets),
+                                            _ptr(kept_idx), _ptr(kept_cnt), _stream()), "tri_select_budgets")
+            return
         _check(lib().tri_select(self._h, _ptr(scores), _ptr(seq_lens), S, n_max, budget, _ptr(kept_idx),
                                 _ptr(kept_cnt), _ptr(ws), 0 if ws is None else ws.numel(), _stream()), "tri_select")
 
@@ -290,7 +302,8 @@ class TriContext:
 
     def compress(self, src: CacheView, cur_pos: torch.Tensor, budget: int, dst: CacheView, ws: torch.Tensor,
                  kept_idx: Optional[torch.Tensor] = None, kept_cnt: Optional[torch.Tensor] = None,
-                 new_seq_lens: Optional[torch.Tensor] = None, device_status: Optional[torch.Tensor] = None):
+                 new_seq_lens: Optional[torch.Tensor] = None, device_status: Optional[torch.Tensor] = None,
+                 unit_budgets: Optional[torch.Tensor] = None):
         S = cur_pos.shape[0]
         cs, cd = src.c_view(), dst.c_view()
         assert cur_pos.dtype == torch.int64
@@ -298,9 +311,28 @@ class TriContext:
             assert kept_idx.dtype == torch.int32 and kept_idx.numel() == self.units(S) * budget
         if kept_cnt is not None:
             assert kept_cnt.dtype == torch.int32 and kept_cnt.numel() == self.units(S)
+        if unit_budgets is not None:
+            assert unit_budgets.dtype == torch.int32 and unit_budgets.numel() == self.units(S) and unit_budgets.is_contiguous()
+            _check(lib().tri_compress_budgets(self._h, ctypes.byref(cs), S, _ptr(cur_pos), budget, _ptr(unit_budgets),
+                                              ctypes.byref(cd), _ptr(kept_idx), _ptr(kept_cnt), _ptr(new_seq_lens),
+                                              _ptr(device_status), _ptr(ws), ws.numel(), _stream()), "tri_compress_budgets")
+            return
         _check(lib().tri_compress(self._h, ctypes.byref(cs), S, _ptr(cur_pos), budget, ctypes.byref(cd),
                                   _ptr(kept_idx), _ptr(kept_cnt), _ptr(new_seq_lens), _ptr(device_status),
                                   _ptr(ws), ws.numel(), _stream()), "tri_compress")
+
+    def compress_windowed(self, src: CacheView, cur_pos: torch.Tensor, budget: int, decoded: torch.Tensor, step: int,
+                          beta: int, dst: CacheView, ws: torch.Tensor, kept_idx: Optional[torch.Tensor] = None,
+                          kept_cnt: Optional[torch.Tensor] = None, new_seq_lens: Optional[torch.Tensor] = None,
+                          device_status: Optional[torch.Tensor] = None):
+        """tri_compress behind the device-side window trigger: sequences whose counter reaches beta and whose cache
+        exceeds the budget are compressed, the others are left alone."""
+        S = cur_pos.shape[0]
+        cs, cd = src.c_view(), dst.c_view()
+        assert cur_pos.dtype == torch.int64 and decoded.dtype == torch.int32 and decoded.numel() == S
+        _check(lib().tri_compress_windowed(self._h, ctypes.byref(cs), S, _ptr(cur_pos), budget, _ptr(decoded), step, beta,
+                                           ctypes.byref(cd), _ptr(kept_idx), _ptr(kept_cnt), _ptr(new_seq_lens),
+                                           _ptr(device_status), _ptr(ws), ws.numel(), _stream()), "tri_compress_windowed")
 
     def compress_host(self, src_host: CacheView, src_dev: CacheView, cur_pos_host: torch.Tensor,
                       cur_pos_dev: torch.Tensor, budget: int, dst_host: CacheView, dst_dev: CacheView,

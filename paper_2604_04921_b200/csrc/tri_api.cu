@@ -224,7 +224,7 @@ namespace {
 
 struct Plan {
     int32_t U, chunk, nchunks;
-    size_t off_E, off_bt, off_bn, off_raw, off_part, off_scores, off_idx, off_cnt, total;
+    size_t off_E, off_bt, off_bn, off_raw, off_part, off_scores, off_idx, off_cnt, off_eff, total;
 };
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -262,6 +262,7 @@ Plan make_plan(const tri_ctx *c, int32_t S, int32_t n_max, int32_t budget, int32
     p.off_scores = o; o += align256((size_t)p.U * n_max * sizeof(float));
     p.off_idx = o;    o += align256((size_t)p.U * (size_t)(budget > 0 ? budget : 0) * sizeof(int32_t));
     p.off_cnt = o;    o += align256((size_t)p.U * sizeof(int32_t));
+    p.off_eff = o;    o += align256((size_t)S * sizeof(int32_t));      // effective lengths of the windowed round
     p.total = o;
     return p;
 }
@@ -453,7 +454,7 @@ tri_status run_fold(tri_ctx *c, int32_t S, const int64_t *cur_pos, char *ws, con
 // round leaves the normalisation to its selection kernel.  The phasors must have been folded (run_fold).
 tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, float *scores,
                      float *raw_out, char *ws, const Plan &pl, int32_t *device_status, cudaStream_t st,
-                     Units un, Layers ly = Layers{0, 0}, int32_t skip_upto = 0)
+                     Units un, Layers ly = Layers{0, 0}, int32_t skip_upto = 0, const int32_t *unit_budgets = nullptr)
 {
     if (ly.count == 0) ly.count = c->desc.n_layers;
     const size_t head0 = (size_t)ly.first * c->desc.n_kv_heads * c->desc.group_size;   // first query head of the range
@@ -465,7 +466,7 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
 
     ScoreParams sp;
     sp.src = to_view(src);
-    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G; sp.u0 = un.first; sp.skip_upto = skip_upto;
+    sp.S = S; sp.H = c->desc.n_kv_heads; sp.G = G; sp.u0 = un.first; sp.skip_upto = skip_upto; sp.unit_budgets = unit_budgets;
     sp.chunk = pl.chunk; sp.nchunks = pl.nchunks;
     sp.E = E; sp.qc = c->qc_d + head0 * kHeadDim; sp.mw = c->mw_d + head0 * kBands;
     sp.bt = (const uint8_t *)(ws + pl.off_bt); sp.bn = (const uint8_t *)(ws + pl.off_bn);
@@ -509,9 +510,10 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
 // score area.
 tri_status run_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
                       int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
-                      Units un, const Plan *pl, char *ws, cudaStream_t st)
+                      Units un, const Plan *pl, char *ws, cudaStream_t st, const int32_t *unit_budgets = nullptr)
 {
     SelectParams p;
+    p.unit_budgets = unit_budgets;
     p.scores = scores; p.scores_w = nullptr; p.seq_lens = seq_lens; p.kept_idx = kept_idx; p.kept_cnt = kept_cnt;
     p.S = S; p.H = c->desc.n_kv_heads; p.n_max = n_max; p.budget = budget; p.u0 = un.first;
     p.raw = nullptr; p.partials = nullptr; p.G = c->desc.group_size; p.chunk = 0; p.nchunks = 0;
@@ -626,18 +628,32 @@ extern "C" tri_status tri_score(tri_ctx *c, const tri_cache_view *src, int32_t S
     return run_score(c, src, S, cur_pos, scores, raw, (char *)ws, pl, nullptr, (cudaStream_t)stream, Units{0, pl.U});
 }
 
-extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S,
-                                 int32_t n_max, int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
-                                 void *ws, size_t ws_bytes, void *stream)
+static tri_status select_impl(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S, int32_t n_max,
+                              int32_t budget, const int32_t *unit_budgets, int32_t *kept_idx, int32_t *kept_cnt, void *stream)
 {
-    (void)ws; (void)ws_bytes;   // the selection keeps its histograms and candidates in shared memory
     tri_status r;
     if (!c || !scores || !seq_lens || !kept_idx || !kept_cnt) return TRI_ERR_INVALID_ARG;
     if ((r = check_device(c)) != TRI_OK) return r;
     if ((r = check_common(c, S, n_max, budget)) != TRI_OK) return r;
     int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
     return run_select(c, scores, seq_lens, S, n_max, budget, kept_idx, kept_cnt, Units{0, U}, nullptr, nullptr,
-                      (cudaStream_t)stream);
+                      (cudaStream_t)stream, unit_budgets);
+}
+
+extern "C" tri_status tri_select(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S,
+                                 int32_t n_max, int32_t budget, int32_t *kept_idx, int32_t *kept_cnt,
+                                 void *ws, size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;   // the selection keeps its histograms and candidates in shared memory
+    return select_impl(c, scores, seq_lens, S, n_max, budget, nullptr, kept_idx, kept_cnt, stream);
+}
+
+extern "C" tri_status tri_select_budgets(tri_ctx *c, const float *scores, const int32_t *seq_lens, int32_t S,
+                                         int32_t n_max, int32_t budget, const int32_t *unit_budgets, int32_t *kept_idx,
+                                         int32_t *kept_cnt, void *stream)
+{
+    if (!unit_budgets) return TRI_ERR_INVALID_ARG;
+    return select_impl(c, scores, seq_lens, S, n_max, budget, unit_budgets, kept_idx, kept_cnt, stream);
 }
 
 extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx,
@@ -661,7 +677,7 @@ extern "C" tri_status tri_compact(tri_ctx *c, const tri_cache_view *src, const i
 static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                                   int32_t budget, const tri_cache_view *dst, int32_t *kept_idx, int32_t *kept_cnt,
                                   int32_t *new_seq_lens, int32_t *device_status, void *ws, size_t ws_bytes,
-                                  cudaStream_t st, int ranges)
+                                  cudaStream_t st, int ranges, const int32_t *unit_budgets = nullptr)
 {
     tri_status r;
     NvtxRange whole("tri_compress");
@@ -677,17 +693,21 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
         {
             NvtxRange part("tri_compress: score");
             // sequences that do not exceed the budget are kept whole: their keys are not even read
-            if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, all, ly, budget)) != TRI_OK) return r;
+            if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, all, ly, budget, unit_budgets)) != TRI_OK) return r;
         }
         {
             NvtxRange part("tri_compress: normalise + select");
-            if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, all, &pl, w, st)) != TRI_OK)
+            if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, all, &pl, w, st, unit_budgets)) != TRI_OK)
                 return r;
         }
         // new_seq_lens may be the very array the scoring and selection kernels read the lengths from, so only the
         // last launch of the round (the gather, which reads kept counts, never lengths) stores it
         NvtxRange part("tri_compress: compact");
-        return run_compact(c, src, idx, cnt, S, budget, dst, new_seq_lens, device_status, all, st);
+        if (!unit_budgets || !new_seq_lens) return run_compact(c, src, idx, cnt, S, budget, dst, new_seq_lens, device_status, all, st);
+        // per-unit budgets: the units of a sequence keep different numbers of rows; the sequence's entry is the largest
+        if ((r = run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, all, st)) != TRI_OK) return r;
+        k_store_max_lens<<<(S + 255) / 256, 256, 0, st>>>(cnt, new_seq_lens, ly.count, S, c->desc.n_kv_heads);
+        return check_launch("k_store_max_lens");
     }
     // Pipelined: the caller's stream scores range after range; behind each range an event lets the side stream
     // select and compact it while the next range is being scored.  The caller's stream waits for the side stream
@@ -697,26 +717,26 @@ static tri_status compress_layers(tri_ctx *c, Layers ly, const tri_cache_view *s
         const int32_t a = (int32_t)((int64_t)pl.U * i / ranges), b = (int32_t)((int64_t)pl.U * (i + 1) / ranges);
         const Units un{a, b - a};
         if (un.count == 0) continue;
-        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, un, ly, budget)) != TRI_OK) return r;
+        if ((r = run_score(c, src, S, cur_pos, nullptr, nullptr, w, pl, device_status, st, un, ly, budget, unit_budgets)) != TRI_OK) return r;
         TRI_CUDA(cudaEventRecord(c->scored[i], st));
         TRI_CUDA(cudaStreamWaitEvent(c->side, c->scored[i], 0));
-        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, un, &pl, w, c->side)) != TRI_OK) return r;
+        if ((r = run_select(c, nullptr, src->seq_lens, S, src->n_max, budget, idx, cnt, un, &pl, w, c->side, unit_budgets)) != TRI_OK) return r;
         if ((r = run_compact(c, src, idx, cnt, S, budget, dst, nullptr, device_status, un, c->side)) != TRI_OK) return r;
     }
     TRI_CUDA(cudaEventRecord(c->side_done, c->side));
     TRI_CUDA(cudaStreamWaitEvent(st, c->side_done, 0));
     if (new_seq_lens) {
         // after every kernel that reads the lengths (new_seq_lens may be that very array)
-        k_store_lens<<<(S + 255) / 256, 256, 0, st>>>(src->seq_lens, new_seq_lens, S, src->n_max, budget);
+        if (unit_budgets) k_store_max_lens<<<(S + 255) / 256, 256, 0, st>>>(cnt, new_seq_lens, ly.count, S, c->desc.n_kv_heads);
+        else k_store_lens<<<(S + 255) / 256, 256, 0, st>>>(src->seq_lens, new_seq_lens, S, src->n_max, budget);
         return check_launch("k_store_lens");
     }
     return TRI_OK;
 }
 
-extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
-                                   int32_t budget, const tri_cache_view *dst, int32_t *kept_idx,
-                                   int32_t *kept_cnt, int32_t *new_seq_lens, int32_t *device_status,
-                                   void *ws, size_t ws_bytes, void *stream)
+static tri_status compress_impl(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos, int32_t budget,
+                                const int32_t *unit_budgets, const tri_cache_view *dst, int32_t *kept_idx, int32_t *kept_cnt,
+                                int32_t *new_seq_lens, int32_t *device_status, void *ws, size_t ws_bytes, void *stream)
 {
     tri_status r;
     if (!c || !cur_pos || !ws) return TRI_ERR_INVALID_ARG;
@@ -729,7 +749,60 @@ extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_
     if ((uintptr_t)ws & 255) return TRI_ERR_INVALID_ARG;
     const int32_t U = c->desc.n_layers * S * c->desc.n_kv_heads;
     return compress_layers(c, Layers{0, c->desc.n_layers}, src, S, cur_pos, budget, dst, kept_idx, kept_cnt, new_seq_lens,
-                           device_status, ws, ws_bytes, (cudaStream_t)stream, pick_ranges(c, U));
+                           device_status, ws, ws_bytes, (cudaStream_t)stream, pick_ranges(c, U), unit_budgets);
+}
+
+extern "C" tri_status tri_compress(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                   int32_t budget, const tri_cache_view *dst, int32_t *kept_idx,
+                                   int32_t *kept_cnt, int32_t *new_seq_lens, int32_t *device_status,
+                                   void *ws, size_t ws_bytes, void *stream)
+{
+    return compress_impl(c, src, S, cur_pos, budget, nullptr, dst, kept_idx, kept_cnt, new_seq_lens, device_status, ws, ws_bytes,
+                         stream);
+}
+
+extern "C" tri_status tri_compress_budgets(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                           int32_t budget, const int32_t *unit_budgets, const tri_cache_view *dst,
+                                           int32_t *kept_idx, int32_t *kept_cnt, int32_t *new_seq_lens,
+                                           int32_t *device_status, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!unit_budgets) return TRI_ERR_INVALID_ARG;
+    return compress_impl(c, src, S, cur_pos, budget, unit_budgets, dst, kept_idx, kept_cnt, new_seq_lens, device_status, ws,
+                         ws_bytes, stream);
+}
+
+extern "C" tri_status tri_compress_windowed(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
+                                            int32_t budget, int32_t *decoded, int32_t step, int32_t beta,
+                                            const tri_cache_view *dst, int32_t *kept_idx, int32_t *kept_cnt,
+                                            int32_t *new_seq_lens, int32_t *device_status, void *ws, size_t ws_bytes,
+                                            void *stream)
+{
+    if (!c || !src || !decoded || step < 0 || beta <= 0 || !ws || ((uintptr_t)ws & 255) || S <= 0 || !src->seq_lens)
+        return TRI_ERR_INVALID_ARG;
+    Plan pl = make_plan(c, S, src->n_max > 0 ? src->n_max : 1, budget);
+    if (ws_bytes < pl.total) return TRI_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t *eff = (int32_t *)((char *)ws + pl.off_eff);
+    tri_cache_view due = *src;
+    due.seq_lens = eff;
+    // argument checks of the round itself, before the counters are touched
+    tri_status r;
+    if ((r = check_device(c)) != TRI_OK) return r;
+    if ((r = check_view(src, true)) != TRI_OK) return r;
+    if ((r = check_view(dst, false)) != TRI_OK) return r;
+    if ((r = check_common(c, S, src->n_max, budget)) != TRI_OK) return r;
+    if (dst->n_max < budget && dst->n_max < src->n_max) return TRI_ERR_INVALID_ARG;
+    if (src->k_kind != dst->k_kind) return TRI_ERR_INVALID_ARG;
+    k_window_begin<<<(S + 255) / 256, 256, 0, st>>>(src->seq_lens, decoded, eff, S, step, beta, budget);
+    if ((r = check_launch("k_window_begin")) != TRI_OK) return r;
+    if ((r = compress_impl(c, &due, S, cur_pos, budget, nullptr, dst, kept_idx, kept_cnt, nullptr, device_status, ws, ws_bytes,
+                           stream)) != TRI_OK)
+        return r;
+    if (new_seq_lens) {
+        k_window_end<<<(S + 255) / 256, 256, 0, st>>>(src->seq_lens, eff, new_seq_lens, S, src->n_max, budget);
+        return check_launch("k_window_end");
+    }
+    return TRI_OK;
 }
 
 extern "C" tri_status tri_set_pipeline(tri_ctx *c, int32_t ranges)

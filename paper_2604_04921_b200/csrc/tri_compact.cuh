@@ -306,4 +306,39 @@ __global__ void k_store_lens(const int32_t *seq_lens, int32_t *new_seq_lens, int
     if (s < S) new_seq_lens[s] = min(min(seq_lens[s], n_max), budget);
 }
 
+// With per-unit budgets the units of a sequence keep different numbers of rows: new_seq_lens[s] is the largest.
+__global__ void k_store_max_lens(const int32_t *kept_cnt, int32_t *new_seq_lens, int32_t L, int32_t S, int32_t H)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    int m = 0;
+    for (int l = 0; l < L; ++l)
+        for (int h = 0; h < H; ++h) m = max(m, kept_cnt[((int64_t)l * S + s) * H + h]);
+    new_seq_lens[s] = m;
+}
+
+// Window trigger of Section 4.3 on the device.  `decoded[s]` counts the tokens a sequence has decoded since its last
+// window boundary; a call adds `step` to it.  At a boundary (count >= beta) the count starts over, and the sequence is
+// due for a round if its cache exceeds the budget.  eff_lens[s] = seq_lens[s] for due sequences and 0 for the others,
+// which every kernel of the round reads as "nothing cached": no key is scored, no row moves.
+__global__ void k_window_begin(const int32_t *seq_lens, int32_t *decoded, int32_t *eff_lens, int32_t S, int32_t step,
+                               int32_t beta, int32_t budget)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= S) return;
+    int c = decoded[s] + step;
+    const bool boundary = c >= beta;
+    if (boundary) c = 0;
+    decoded[s] = c;
+    eff_lens[s] = (boundary && seq_lens[s] > budget) ? seq_lens[s] : 0;
+}
+
+// After the round: due sequences shrink to the budget, the others keep their length (the two arrays may be one).
+__global__ void k_window_end(const int32_t *seq_lens, const int32_t *eff_lens, int32_t *new_seq_lens, int32_t S,
+                             int32_t n_max, int32_t budget)
+{
+    const int s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < S) new_seq_lens[s] = eff_lens[s] > 0 ? min(min(eff_lens[s], n_max), budget) : seq_lens[s];
+}
+
 }  // namespace tri

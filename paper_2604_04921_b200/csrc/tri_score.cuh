@@ -93,6 +93,7 @@ struct ScoreParams {
     int32_t S, H, G;
     int32_t u0;           // first unit of this launch (a round may be issued as several launches over unit ranges)
     int32_t skip_upto;    // units of at most this many keys are not scored (the fused round keeps them whole); 0 = score all
+    const int32_t *unit_budgets;   // [U] or NULL: with skip_upto > 0, the per-unit value min(unit_budgets[u], skip_upto) applies
     int32_t chunk;        // keys per block (multiple of 16)
     int32_t nchunks;      // blocks per unit
     const double2 *E;     // [S][64]  e^{i omega_f p_q} Dbar_f
@@ -104,6 +105,12 @@ struct ScoreParams {
     double2 *partials;    // [U][nchunks][G]  (sum, sum of squares) of raw over the block's keys
     int32_t *device_status;
 };
+
+// Units of at most this many keys are left unscored by the fused round (it keeps them whole).
+__device__ __forceinline__ int skip_limit(const ScoreParams &p, int u)
+{
+    return (p.unit_budgets && p.skip_upto > 0) ? min(max(__ldg(p.unit_budgets + u), 0), p.skip_upto) : p.skip_upto;
+}
 
 // ---------------------------------------------------------------------------------------
 // Raw scoring of fp32 pre-RoPE keys (k_kind 1): the reference-style slow path, all in double.
@@ -121,7 +128,7 @@ k_score_f32_pre(const ScoreParams p, const double *__restrict__ omega, const dou
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int n = min(__ldg(p.src.seq_lens + s), p.src.n_max);
     const int key_begin = chunk * p.chunk;
-    if (key_begin >= n || n <= p.skip_upto) return;
+    if (key_begin >= n || n <= skip_limit(p, u)) return;
     const int key_end = min(key_begin + p.chunk, n);
     const int G = p.G;
     const int64_t pq = cur_pos[s];

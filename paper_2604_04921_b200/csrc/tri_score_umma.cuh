@@ -204,7 +204,7 @@ k_score_umma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int n = min(__ldg(p.src.seq_lens + s), p.src.n_max);
     const int key_begin = chunk * p.chunk;
-    if (key_begin >= n || n <= p.skip_upto) return;
+    if (key_begin >= n || n <= skip_limit(p, u)) return;
     const int key_end = min(key_begin + p.chunk, n);
     const int G = p.G;
     const int ntiles = (key_end - key_begin + kUTile - 1) / kUTile;

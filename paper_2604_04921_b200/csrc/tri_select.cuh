@@ -35,6 +35,7 @@ struct SelectParams {
     int32_t *kept_cnt;        // [U]
     int32_t S, H, n_max, budget;
     int32_t u0;               // first unit of this launch
+    const int32_t *unit_budgets;   // [U] or NULL: per-unit budget, clamped to [0, budget]
     // FUSED only: raw scores and partial sums of the scoring kernel
     const float *raw;         // [U][n_max][G]
     const double2 *partials;  // [U][nchunks][G]
@@ -117,10 +118,11 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
     const int n = min(__ldg(p.seq_lens + s), p.n_max);
     const float *sc = p.scores + (int64_t)u * p.n_max;
     int32_t *out = p.kept_idx + (int64_t)u * p.budget;
-    const int cnt = min(n, p.budget);
+    const int budget = p.unit_budgets ? min(max(__ldg(p.unit_budgets + u), 0), p.budget) : p.budget;
+    const int cnt = min(n, budget);
     if (tid == 0) p.kept_cnt[u] = cnt;
-    if (n <= p.budget) {                        // the cache does not exceed the budget: keep all
-        for (int i = tid; i < n; i += kSelThreads) out[i] = i;
+    if (n <= budget || budget == 0) {           // the cache does not exceed the budget: keep all (or nothing is kept)
+        for (int i = tid; i < cnt; i += kSelThreads) out[i] = i;
         return;
     }
 
@@ -158,7 +160,7 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
         for (int i = tid; i < n; i += kSelThreads) atomicAdd(&hist[value_bin(sc[i])], 1u);
     }
     __syncthreads();                            // histogram complete; parked scores visible to the whole block
-    find_bin<THREADS>(hist, (uint32_t)p.budget, warp_sums, &sel_bin, &sel_need);
+    find_bin<THREADS>(hist, (uint32_t)budget, warp_sums, &sel_bin, &sel_need);
     const uint32_t vb = sel_bin;
     uint32_t need = sel_need;                   // keys still to take from value bin vb
 
@@ -208,7 +210,7 @@ __global__ void __launch_bounds__(THREADS, 2048 / THREADS) k_select(const Select
     // ---- emit kept slots in ascending order; among keys equal to T the lowest slots win ----
     // J keys per thread and span (at most 32, fewer for short units so that no sweep runs empty)
     const int J = min(32, (n + kSelThreads - 1) / kSelThreads);
-    const bool dense = 2 * p.budget > n;        // more than half of the keys are kept
+    const bool dense = 2 * budget > n;        // more than half of the keys are kept
     uint32_t base = 0, need_rem = need;
 #pragma unroll 1
     for (int span = 0; span < n; span += kSelThreads * J) {

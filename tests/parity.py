@@ -90,7 +90,7 @@ def check_compacted(k_out, v_out, pos_out, idx_gpu: np.ndarray, ref: dict):
 
 
 def run_compress(w: W.Workload, budget: int, ctx: tb.TriContext = None, in_place: bool = False,
-                 want_scores: bool = True):
+                 want_scores: bool = True, unit_budgets=None):
     """tri_score (+raw) and tri_compress on the whole workload.  Returns a dict of device tensors."""
     sp = w.spec
     own = ctx is None
@@ -124,7 +124,7 @@ def run_compress(w: W.Workload, budget: int, ctx: tb.TriContext = None, in_place
         dst = tb.CacheView(k2, v2, positions=p2)
         out["k_out"], out["v_out"], out["pos_out"] = k2, v2, p2
     ctx.compress(src, w.cur_pos, budget, dst, ws, kept_idx=kept_idx, kept_cnt=kept_cnt, new_seq_lens=new_lens,
-                 device_status=status)
+                 device_status=status, unit_budgets=unit_budgets)
     torch.cuda.synchronize()
     out.update(kept_idx=kept_idx, kept_cnt=kept_cnt, new_seq_lens=new_lens, status=status, ctx=ctx)
     if own:

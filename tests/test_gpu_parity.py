@@ -364,6 +364,51 @@ def test_lengths_updated_in_place_with_many_units():
         check_unit(w, res, oracle_unit(w, l, s, h, B), l, s, h, B)
 
 
+@pytest.mark.parametrize("kind", ["contiguous", "paged_in_place"])
+def test_budget_per_unit(kind):
+    """Head-specific budgets (the future work of Appendix A): every (layer, sequence, head) keeps its own number of
+    rows, drawn in [B/4, B], with a few units at 0, at 1 and above their length.  Every unit against the oracle run
+    with that unit's budget; tri_select_budgets on the exported scores gives the same indices."""
+    if kind == "contiguous":
+        sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="ub", n_layers=2, n_kv_heads=3, n_seqs=2, n_keys=3000, budget=512)
+    else:
+        sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name="ub_p", n_layers=2, n_kv_heads=2, n_seqs=3, n_keys=2500,
+                                                      n_keys_min=600, budget=512)
+    w = W.make_workload(sp, DEV)
+    B, L, S, H = sp.budget, sp.n_layers, sp.n_seqs, sp.n_kv_heads
+    U = L * S * H
+    g = torch.Generator().manual_seed(3)
+    ub = torch.randint(B // 4, B + 1, (U,), generator=g, dtype=torch.int32)
+    ub[1], ub[2], ub[U - 1], ub[U - 2] = 0, 1, 10 ** 6, -5          # nothing, one row, clamped to B, negative = nothing
+    ub_d = ub.to(DEV)
+    refs = {}
+    for (l, s_, h) in _all_units(w):
+        b_u = int(min(max(int(ub[unit_index(w, l, s_, h)]), 0), B))
+        refs[(l, s_, h)] = (b_u, oracle_unit(w, l, s_, h, max(b_u, 1)))
+    res = run_compress(w, B, in_place=(kind != "contiguous"), unit_budgets=ub_d)
+    assert int(res["status"].item()) == 0
+    lens = w.seq_lens.tolist()
+    per_seq = [0] * S
+    for (l, s_, h), (b_u, ref) in refs.items():
+        u = unit_index(w, l, s_, h)
+        cnt = int(res["kept_cnt"][u])
+        assert cnt == min(b_u, lens[s_])
+        per_seq[s_] = max(per_seq[s_], cnt)
+        if b_u == 0:
+            continue
+        check_unit(w, res, ref, l, s_, h, b_u)
+    assert res["new_seq_lens"].tolist() == per_seq
+    # selection alone, from the scores the round exported
+    idx = torch.full((U, B), -1, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(U, dtype=torch.int32, device=DEV)
+    n_max = res["scores"].shape[1]
+    res["ctx"].select(res["scores"], w.seq_lens, n_max, B, idx, cnt, unit_budgets=ub_d)
+    torch.cuda.synchronize()
+    assert torch.equal(cnt, res["kept_cnt"])
+    valid = torch.arange(B, device=DEV)[None, :] < cnt[:, None]
+    assert torch.equal(idx[valid], res["kept_idx"][valid])
+
+
 def test_only_overflowing_sequences_are_touched():
     """A batch in which one sequence exceeds the budget and two do not: the short ones are kept whole, in order,
     and the round gives the same kept rows for the long one as a batch holding it alone."""
@@ -584,6 +629,91 @@ def test_round_replays_from_a_cuda_graph():
     torch.cuda.synchronize()
     assert torch.equal(idx, later["kept_idx"]) and not torch.equal(idx, direct["kept_idx"])
     assert torch.equal(v2.view(torch.int16), later["v_out"].view(torch.int16))
+
+
+def test_windowed_round_in_a_decode_loop_from_a_graph():
+    """tri_compress_windowed captured once and replayed after every decoded token (Section 4.3's trigger on the device):
+    nothing moves until a sequence's window counter reaches beta with its cache above the budget; then that sequence
+    alone is compressed in place.  Two sequences out of phase (one starts at the budget, one far below it), 40 steps,
+    against a host model that applies the oracle at the same moments."""
+    B, beta, steps, S, H = 64, 8, 40, 2, 2
+    cap = B + beta
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="win", n_layers=1, n_kv_heads=H, n_seqs=S, n_keys=B + steps, budget=B)
+    full = W.make_workload(sp, DEV)                     # every token either sequence will ever hold: slot i = position i
+    G = sp.group_size
+    start = [B, 30]
+    k = torch.zeros(1, S, H, cap, 128, dtype=torch.bfloat16, device=DEV); v = torch.zeros_like(k)
+    pos = torch.zeros(1, S, H, cap, dtype=torch.int32, device=DEV)
+    lens = torch.tensor(start, dtype=torch.int32, device=DEV)
+    cur = torch.tensor(start, dtype=torch.int64, device=DEV)
+    decoded = torch.zeros(S, dtype=torch.int32, device=DEV)
+    cnt = torch.zeros(S * H, dtype=torch.int32, device=DEV)
+    host = {}
+    for s_ in range(S):
+        n0 = start[s_]
+        k[0, s_, :, :n0], v[0, s_, :, :n0] = full.k[0, s_, :, :n0], full.v[0, s_, :, :n0]
+        pos[0, s_, :, :n0] = torch.arange(n0, dtype=torch.int32, device=DEV)
+        for h in range(H):
+            host[(s_, h)] = dict(k=full.k[0, s_, h, :n0].cpu(), v=full.v[0, s_, h, :n0].cpu(), pos=torch.arange(n0))
+    ctx = make_ctx(full)
+    ws = ctx.workspace(S, cap, B)
+    view = tb.CacheView(k, v, seq_lens=lens, positions=pos)
+    ctx.compress_windowed(view, cur, B, decoded, 0, beta, view, ws, kept_cnt=cnt, new_seq_lens=lens)   # set-up call, nothing due
+    torch.cuda.synchronize()
+    assert lens.tolist() == start and decoded.tolist() == [0, 0]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.compress_windowed(view, cur, B, decoded, 1, beta, view, ws, kept_cnt=cnt, new_seq_lens=lens)
+    h_len, h_dec, rounds = list(start), [0, 0], 0
+    for step in range(steps):
+        for s_ in range(S):                            # the model appends one token per sequence
+            t = start[s_] + step
+            n = h_len[s_]
+            k[0, s_, :, n], v[0, s_, :, n] = full.k[0, s_, :, t], full.v[0, s_, :, t]
+            pos[0, s_, :, n] = t
+            for h in range(H):
+                st = host[(s_, h)]
+                host[(s_, h)] = dict(k=torch.cat([st["k"], full.k[0, s_, h, t:t + 1].cpu()]),
+                                     v=torch.cat([st["v"], full.v[0, s_, h, t:t + 1].cpu()]), pos=torch.cat([st["pos"], torch.tensor([t])]))
+            h_len[s_] += 1
+        lens.copy_(torch.tensor(h_len, dtype=torch.int32))
+        cur.copy_(torch.tensor([start[s_] + step + 1 for s_ in range(S)], dtype=torch.int64))
+        graph.replay()
+        torch.cuda.synchronize()
+        for s_ in range(S):
+            h_dec[s_] += 1
+            due = False
+            if h_dec[s_] >= beta:
+                h_dec[s_] = 0
+                due = h_len[s_] > B
+            for h in range(H):
+                st = host[(s_, h)]
+                if due:
+                    _, s_o, idx_o = oracle.unit_bf16(W.bf16_bits(st["k"]), st["pos"].numpy(), start[s_] + step + 1,
+                                                     full.q_center[0, h * G:(h + 1) * G].double().numpy(),
+                                                     full.q_mean_norm[0, h * G:(h + 1) * G].double().numpy(), B, theta=sp.theta)
+                    got_pos = pos[0, s_, h, :B].cpu().long()
+                    want_pos = st["pos"][torch.from_numpy(idx_o.astype(np.int64))]
+                    if not torch.equal(got_pos, want_pos):
+                        diff = np.setxor1d(got_pos.numpy(), want_pos.numpy())
+                        s_b = np.sort(s_o)[::-1][B - 1]
+                        assert np.all(np.abs(s_o[np.isin(st["pos"].numpy(), diff)] - s_b) <= 1e-3 * max(1.0, abs(s_b)))
+                    sel = torch.from_numpy(np.searchsorted(st["pos"].numpy(), got_pos.numpy()))
+                    assert torch.equal(st["pos"][sel], got_pos)
+                    host[(s_, h)] = dict(k=st["k"][sel], v=st["v"][sel], pos=got_pos)
+                    assert int(cnt[s_ * H + h]) == B
+                    rounds += 1
+                else:
+                    assert int(cnt[s_ * H + h]) == 0
+                st = host[(s_, h)]
+                n = st["pos"].shape[0]
+                assert torch.equal(pos[0, s_, h, :n].cpu().long(), st["pos"])
+                assert torch.equal(k[0, s_, h, :n].cpu().view(torch.int16), st["k"].view(torch.int16))
+                assert torch.equal(v[0, s_, h, :n].cpu().view(torch.int16), st["v"].view(torch.int16))
+            if due:
+                h_len[s_] = B
+        assert lens.tolist() == h_len and decoded.tolist() == h_dec, step
+    assert rounds >= 2 * H * 3                         # both sequences were compressed several times
 
 
 def test_bad_page_id_sets_status_not_fault():
