@@ -242,6 +242,8 @@ tri_status tri_compress_host(tri_ctx *ctx, const tri_cache_view *src_host, const
  *     with events.
  */
 #define TRI_SCORE_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+/* Bytes of the built-in array a call of tri_score_static with this shape would use (0 for bad arguments). */
+size_t tri_score_static_bytes(const tri_ctx *ctx, int32_t S, int32_t n_max);
 tri_status tri_score_static(tri_ctx *ctx, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                             float *scores, float *raw, void *stream);
 

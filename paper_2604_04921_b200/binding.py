@@ -24,7 +24,7 @@ HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cu
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",
-           "tri_compress", "tri_select_budgets", "tri_compress_budgets", "tri_compress_windowed", "tri_compress_host", "tri_score_static", "tri_compress_launches", "tri_set_pipeline", "tri_set_score_kernel", "tri_last_cuda_error",
+           "tri_compress", "tri_select_budgets", "tri_compress_budgets", "tri_compress_windowed", "tri_compress_host", "tri_score_static", "tri_score_static_bytes", "tri_compress_launches", "tri_set_pipeline", "tri_set_score_kernel", "tri_last_cuda_error",
            "tri_profile_begin", "tri_profile_read", "tri_profile_end",
            "tri_calib_state_bytes", "tri_calib_workspace_bytes", "tri_calib_reset", "tri_calib_accumulate",
            "tri_calib_finalize", "tri_selftest_bounded_wait"]
@@ -97,6 +97,8 @@ def lib():
     L.tri_score.restype = ctypes.c_int
     L.tri_score_static.argtypes = [P, VP, i32, P, P, P, P]
     L.tri_score_static.restype = ctypes.c_int
+    L.tri_score_static_bytes.argtypes = [P, i32, i32]
+    L.tri_score_static_bytes.restype = sz
     L.tri_select.argtypes = [P, P, P, i32, i32, i32, P, P, P, sz, P]
     L.tri_select.restype = ctypes.c_int
     L.tri_compact.argtypes = [P, VP, P, P, i32, i32, VP, P, P]
@@ -256,6 +258,10 @@ class TriContext:
                                ws.numel(), _stream()), "tri_score")
 
     STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+    def score_static_bytes(self, S: int, n_max: int) -> int:
+        """Bytes of the built-in array score_static would use for this shape."""
+        return int(lib().tri_score_static_bytes(self._h, S, n_max))
 
     def score_static(self, src: CacheView, cur_pos: torch.Tensor, scores: torch.Tensor,
                      raw: Optional[torch.Tensor] = None):

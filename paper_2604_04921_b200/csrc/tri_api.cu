@@ -1003,6 +1003,12 @@ static tri_status score_scratch_address(int dev, void **out)
     return TRI_OK;
 }
 
+extern "C" size_t tri_score_static_bytes(const tri_ctx *c, int32_t S, int32_t n_max)
+{
+    if (!c || S <= 0 || n_max <= 0) return 0;
+    return make_plan(c, S, n_max, 0).off_scores;    // phasors (+ folded operands) + raw scores + partial sums
+}
+
 extern "C" tri_status tri_score_static(tri_ctx *c, const tri_cache_view *src, int32_t S, const int64_t *cur_pos,
                                        float *scores, float *raw, void *stream)
 {

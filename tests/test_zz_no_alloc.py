@@ -70,11 +70,13 @@ def test_static_scratch_scoring_matches_tri_score_twice_in_a_row():
 
 
 def _scratch_need(ctx, S, U, n_max):
-    """Bytes of the built-in array a shape uses: the documented workspace of tri_score minus its final-score
-    area (U * n_max floats) and its kept-count area (U ints), which tri_score_static does not need; every area
-    is rounded up to 256 bytes."""
-    up = lambda x: (x + 255) // 256 * 256
-    return ctx.workspace_bytes(S, n_max, 0) - up(U * n_max * 4) - up(U * 4)
+    """Bytes of the built-in array a shape uses, as the library states them; checked here against the header's
+    account of what goes there (1 KiB of phasors per sequence, 4 G bytes of raw scores per key, 16 G bytes of partial
+    sums per scoring block of at least 1,024 keys, each area rounded up to 256 bytes; G = 4 here)."""
+    need = ctx.score_static_bytes(S, n_max)
+    raw = U * n_max * 16
+    assert raw + 1024 * S <= need <= raw + 1024 * S + U * (n_max // 1024 + 1) * 64 + 3 * 256
+    return need
 
 
 def test_static_scratch_limit_is_exact():
