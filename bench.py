@@ -43,12 +43,12 @@ OTHER_WORKLOADS = (("qwen3_8b_steady_b64", 0), ("qwen3_8b_oneshot_32k", 0), ("qw
 NOMINAL_HBM_GBS = 8000.0
 
 
-# DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum per key),
-# valid only for the kernel source it was taken on.
-SCORE_TRAFFIC = {"bytes_per_key": (268564992 + 13988352) / 1048576,
+# DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum of one launch of
+# k_score_tma<1,0> on 1,048,576 keys: 268,499,200 B + 14,236,928 B), valid only for the kernel source it was taken on.
+SCORE_TRAFFIC = {"bytes_per_key": (268499200 + 14236928) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
-                 "sha256": "f732a90f8607130c89fe05b59d9091a3e58e1ac37d4ac1008fe7c2a7f99acfa7"}
+                 "sha256": "09de78855e1affb1a48f05f07ba6eacd415f15845f53292a8431f791b9374d0e"}
 
 
 def score_traffic_per_launch(keys):
