@@ -285,7 +285,7 @@ def run_calibration(args):
 class Round:
     """One workload resident on the device with everything a timed tri_compress step needs."""
 
-    def __init__(self, spec, L, dev):
+    def __init__(self, spec, L, dev, pre_rope=False):
         import torch
         from paper_2604_04921_b200 import binding as tb
         from paper_2604_04921_b200 import workloads as W
@@ -293,18 +293,19 @@ class Round:
         self.w = w = W.make_workload(spec, dev, layer0=0, n_layers=L)
         S, H, G, B = spec.n_seqs, spec.n_kv_heads, spec.group_size, spec.budget
         self.ctx = tb.TriContext(L, H, G, w.q_center, w.q_mean_norm, rope_theta=spec.theta)
-        self.src = tb.CacheView(w.k, w.v, seq_lens=w.seq_lens, positions=w.positions, page_table=w.page_table)
+        # pre_rope: the same bf16 rows read as pre-RoPE vectors (k_kind 2): the kernels' work does not depend on the values
+        self.src = tb.CacheView(w.k, w.v, seq_lens=w.seq_lens, positions=w.positions, page_table=w.page_table, pre_rope=pre_rope)
         self.n_max = self.src.c_view().n_max
         self.U = L * S * H
         if w.paged:
             # compacted rows are written back into the sequence's own pages (in place)
-            self.dst = tb.CacheView(w.k, w.v, page_table=w.page_table, n_max=self.n_max)
+            self.dst = tb.CacheView(w.k, w.v, page_table=w.page_table, n_max=self.n_max, pre_rope=pre_rope)
             self.k2 = self.v2 = self.p2 = None
         else:
             self.k2 = torch.empty(L, S, H, B, 128, dtype=torch.bfloat16, device=dev)
             self.v2 = torch.empty_like(self.k2)
             self.p2 = torch.empty(L, S, H, B, dtype=torch.int32, device=dev)
-            self.dst = tb.CacheView(self.k2, self.v2, positions=self.p2)
+            self.dst = tb.CacheView(self.k2, self.v2, positions=self.p2, pre_rope=pre_rope)
         self.ws = self.ctx.workspace(S, self.n_max, B, dev)
         self.kept_cnt = torch.zeros(self.U, dtype=torch.int32, device=dev)
         self.lens = w.seq_lens.tolist()
@@ -391,6 +392,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="time the headline workload only")
+    ap.add_argument("--pre-rope", action="store_true", help="treat the bf16 keys as pre-RoPE vectors (k_kind 2: fp32 scoring with phasor tables)")
     ap.add_argument("--calibration", action="store_true", help="time the calibration-statistics pass instead of the round")
     ap.add_argument("--tokens", type=int, default=0, help="--calibration: tokens per pass (default 262,144)")
     args = ap.parse_args()
@@ -400,7 +402,7 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
     from paper_2604_04921_b200 import workloads as W
-    others = args.workload is None and args.layers == 0 and not args.no_others
+    others = args.workload is None and args.layers == 0 and not args.no_others and not args.pre_rope
     spec = W.SPECS[args.workload or DEFAULT_WORKLOAD]
     if args.impl == "reference":
         run_reference(args, spec)
@@ -444,7 +446,7 @@ def main():
         return n, ms, (sampler.summary(first) if rank == 0 else None)
 
     L = args.layers if args.layers > 0 else spec.n_layers
-    rd = Round(spec, L, dev)
+    rd = Round(spec, L, dev, pre_rope=args.pre_rope)
     rd.warm(args.warmup)
     barrier()
     sustained = None
@@ -463,6 +465,8 @@ def main():
     score_bytes = 256 * rd.keys_per_step
     score_gbs = score_bytes / (per["score"] * 1e-3) / 1e9
     cfg = workload_config(spec, L, world)
+    if args.pre_rope:
+        cfg["keys"] = "bf16 pre-RoPE (k_kind 2)"
     line = {
         "metric": METRIC, "value": whole_job_value(world, rd.keys_per_step, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -470,8 +474,8 @@ def main():
         "config": cfg,
         "keys_per_step": rd.keys_per_step,
         "hbm": rd.hbm(ms_step, peak),
-        "roofline": {"kernel": "k_score_tma", "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(rd.keys_per_step), "peak_source": peak_src,
+        "roofline": {"kernel": "k_score_bf16_pre" if args.pre_rope else ("k_score_umma" if spec.group_size > 4 else "k_score_tma"), "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(rd.keys_per_step) if (spec.group_size <= 4 and not args.pre_rope) else None, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"],
                      "note": "per step; a pipelined round issues the scoring as several launches over unit ranges, "
                              "their bytes and durations are summed"},

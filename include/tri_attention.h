@@ -84,10 +84,13 @@ tri_status tri_destroy(tri_ctx *ctx);
  *                           row at  l*stride_layer + page*stride_page + h*stride_head + (n % page_size)*stride_slot
  */
 typedef struct {
-    void *k;                   /* keys: bf16 post-RoPE (k_kind 0) or fp32 pre-RoPE (k_kind 1)   */
+    void *k;                   /* keys: bf16 post-RoPE (k_kind 0), fp32 pre-RoPE (1) or bf16 pre-RoPE (2) */
     void *v;                   /* values, bf16, same strides as k; NULL = no value cache        */
     int32_t k_kind;            /* 0: bf16 as cached by the model (post-RoPE) -- the fast path
-                                  1: fp32 pre-RoPE vectors (needs `positions` or slot = position) */
+                                  1: fp32 pre-RoPE vectors, scored in double (a slow reference-style path)
+                                  2: bf16 pre-RoPE vectors (the k_f of Section 4.1 as they are), scored in fp32 with
+                                     tabulated distance phasors; p_q - p_k must lie in [0, 2^21)
+                                  1 and 2 need `positions`, or slot = position                                   */
     int32_t paged;
     int64_t stride_layer, stride_seq, stride_head, stride_tok;
     const int32_t *page_table; /* device [S][max_pages_per_seq]                                  */

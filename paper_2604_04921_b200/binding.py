@@ -169,6 +169,7 @@ class CacheView:
     positions: Optional[torch.Tensor] = None      # [L, S, H, n_max] int32
     page_table: Optional[torch.Tensor] = None     # [S, max_pages] int32
     n_max: Optional[int] = None
+    pre_rope: bool = False                        # bf16 keys are pre-RoPE vectors (k_kind 2); fp32 keys always are
 
     def c_view(self) -> _CacheView:
         k = self.k
@@ -179,7 +180,7 @@ class CacheView:
         cv = _CacheView()
         cv.k = k.data_ptr()
         cv.v = self.v.data_ptr() if self.v is not None else None
-        cv.k_kind = 0 if k.dtype == torch.bfloat16 else 1
+        cv.k_kind = (2 if self.pre_rope else 0) if k.dtype == torch.bfloat16 else 1
         if self.page_table is None:
             cv.paged = 0
             cv.stride_layer, cv.stride_seq, cv.stride_head, cv.stride_tok = k.stride()[:4]

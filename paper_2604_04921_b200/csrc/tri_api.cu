@@ -33,6 +33,7 @@ struct tri_ctx {
     double2 *dbar_d;     // [64]  (1/|D|) sum_delta e^{i omega_f delta}
     float *qc_d;         // [L][H*G][128]
     float *mw_d;         // [L][H*G][64]   weight of |k_f| in the norm term
+    float2 *rot_lo_d, *rot_hi_d;   // phasor tables of the bf16 pre-RoPE path (see k_score_bf16_pre)
     // tri_profile_begin .. tri_profile_end: an event pair around every launch of tri_compress
     bool profiling;
     ProfRec prof[kMaxProf];
@@ -111,7 +112,7 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
     if (!c) return TRI_ERR_INVALID_ARG;
     c->desc = *desc;
     c->desc.offsets = nullptr;
-    c->omega_d = nullptr; c->dbar_d = nullptr; c->qc_d = nullptr; c->mw_d = nullptr;
+    c->omega_d = nullptr; c->dbar_d = nullptr; c->qc_d = nullptr; c->mw_d = nullptr; c->rot_lo_d = nullptr; c->rot_hi_d = nullptr;
     c->profiling = false;
     c->prof_used = 0;
     c->have_back = false;
@@ -147,6 +148,18 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
                      : desc->norm_variant == 1 ? en : 0.0;
             mw[i * kBands + f] = (float)w;
         }
+    // phasors of query-to-key distances for pre-RoPE bf16 keys: Dbar_f e^{i omega_f b} and e^{i omega_f 512 a}, band-major
+    std::vector<float2> rot_lo((size_t)kBands * kRotLo), rot_hi((size_t)kBands * kRotHi);
+    for (int f = 0; f < kBands; ++f) {
+        for (int b = 0; b < kRotLo; ++b) {
+            const double cs = std::cos(omega[f] * b), sn = std::sin(omega[f] * b);
+            rot_lo[(size_t)f * kRotLo + b] = make_float2((float)(cs * dbar[f].x - sn * dbar[f].y), (float)(cs * dbar[f].y + sn * dbar[f].x));
+        }
+        for (int a = 0; a < kRotHi; ++a) {
+            const double ang = omega[f] * (double)kRotLo * a;
+            rot_hi[(size_t)f * kRotHi + a] = make_float2((float)std::cos(ang), (float)std::sin(ang));
+        }
+    }
     tri_status st = TRI_OK;
     do {
         if ((e = prepare_device()) != cudaSuccess) break;
@@ -158,6 +171,10 @@ extern "C" tri_status tri_create(const tri_model_desc *desc, const float *q_cent
         if ((e = cudaMemcpy(c->dbar_d, dbar, sizeof dbar, cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(c->qc_d, q_center, nq * kHeadDim * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaMemcpy(c->mw_d, mw.data(), nq * kBands * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMalloc(&c->rot_lo_d, rot_lo.size() * sizeof(float2))) != cudaSuccess) break;
+        if ((e = cudaMalloc(&c->rot_hi_d, rot_hi.size() * sizeof(float2))) != cudaSuccess) break;
+        if ((e = cudaMemcpy(c->rot_lo_d, rot_lo.data(), rot_lo.size() * sizeof(float2), cudaMemcpyHostToDevice)) != cudaSuccess) break;
+        if ((e = cudaMemcpy(c->rot_hi_d, rot_hi.data(), rot_hi.size() * sizeof(float2), cudaMemcpyHostToDevice)) != cudaSuccess) break;
         if ((e = cudaStreamCreateWithFlags(&c->back, cudaStreamNonBlocking)) != cudaSuccess) break;
         int made = 0;
         for (; made <= kHostSlabs; ++made)
@@ -213,6 +230,8 @@ extern "C" tri_status tri_destroy(tri_ctx *c)
     cudaFree(c->dbar_d);
     cudaFree(c->qc_d);
     cudaFree(c->mw_d);
+    cudaFree(c->rot_lo_d);
+    cudaFree(c->rot_hi_d);
     delete c;
     return TRI_OK;
 }
@@ -288,7 +307,7 @@ View to_view(const tri_cache_view *v)
 tri_status check_view(const tri_cache_view *v, bool need_lens)
 {
     if (!v || !v->k) return TRI_ERR_INVALID_ARG;
-    if (v->k_kind < 0 || v->k_kind > 1 || v->n_max <= 0) return TRI_ERR_INVALID_ARG;
+    if (v->k_kind < 0 || v->k_kind > 2 || v->n_max <= 0) return TRI_ERR_INVALID_ARG;
     if (need_lens && !v->seq_lens) return TRI_ERR_INVALID_ARG;
     if (((uintptr_t)v->k & 15) || ((uintptr_t)v->v & 15)) return TRI_ERR_INVALID_ARG;
     if (v->stride_layer % 8 || v->stride_head % 8) return TRI_ERR_INVALID_ARG;
@@ -485,6 +504,17 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
                                          : launch_score_tma<1>(NT, grid, st, map, sp);
             if (r != TRI_OK) return r;
         }
+    } else if (src->k_kind == 2) {
+        const int gp = G <= 4 ? 4 : (G <= 8 ? 8 : 16);
+        if (c->desc.pair_layout == 0) {
+            if (gp == 4) k_score_bf16_pre<0, 4><<<grid, kScoreThreads, 0, st>>>(sp, c->rot_lo_d, c->rot_hi_d, cur_pos);
+            else if (gp == 8) k_score_bf16_pre<0, 8><<<grid, kScoreThreads, 0, st>>>(sp, c->rot_lo_d, c->rot_hi_d, cur_pos);
+            else k_score_bf16_pre<0, 16><<<grid, kScoreThreads, 0, st>>>(sp, c->rot_lo_d, c->rot_hi_d, cur_pos);
+        } else {
+            if (gp == 4) k_score_bf16_pre<1, 4><<<grid, kScoreThreads, 0, st>>>(sp, c->rot_lo_d, c->rot_hi_d, cur_pos);
+            else if (gp == 8) k_score_bf16_pre<1, 8><<<grid, kScoreThreads, 0, st>>>(sp, c->rot_lo_d, c->rot_hi_d, cur_pos);
+            else k_score_bf16_pre<1, 16><<<grid, kScoreThreads, 0, st>>>(sp, c->rot_lo_d, c->rot_hi_d, cur_pos);
+        }
     } else {
         if (c->desc.pair_layout == 0)
             k_score_f32_pre<0><<<grid, kScoreThreads, 0, st>>>(sp, c->omega_d, c->dbar_d, cur_pos);
@@ -543,7 +573,7 @@ bool aliases(const tri_cache_view *a, const tri_cache_view *b)
 // Whether the round compacts bf16 K + V in place: then the gather is two launches (tiled prefix, parallel pass).
 bool two_pass_compaction(const tri_cache_view *src, const tri_cache_view *dst)
 {
-    return aliases(src, dst) && src->k_kind == 0 && src->v && dst->v;
+    return aliases(src, dst) && src->k_kind != 1 && src->v && dst->v;
 }
 
 tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx, const int32_t *kept_cnt,
@@ -554,11 +584,11 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
     p.src = to_view(src); p.dst = to_view(dst);
     p.kept_idx = kept_idx; p.kept_cnt = kept_cnt; p.new_seq_lens = new_seq_lens;
     p.S = S; p.H = c->desc.n_kv_heads; p.budget = budget; p.u0 = un.first;
-    p.k_esize = src->k_kind == 0 ? 2 : 4;
+    p.k_esize = src->k_kind == 1 ? 4 : 2;
     p.k_vec = kHeadDim * p.k_esize / 16;
     p.v_vec = (src->v && dst->v) ? kHeadDim * 2 / 16 : 0;
     p.device_status = device_status;
-    const bool rows16 = src->k_kind == 0 && p.v_vec != 0;     // bf16 K and V: the row-gather kernel applies
+    const bool rows16 = src->k_kind != 1 && p.v_vec != 0;     // bf16 K and V: the row-gather kernel applies
     const int U = un.count;
     dim3 grid(U, (budget + kFastRowsPerBlock - 1) / kFastRowsPerBlock);
     const int pr = prof_open(c, 4, st);
@@ -851,7 +881,7 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
     if (src_dev->k_kind != dst_dev->k_kind || !ws || ((uintptr_t)ws & 255)) return TRI_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int L = c->desc.n_layers, H = c->desc.n_kv_heads;
-    const size_t kes = src_host->k_kind == 0 ? 2 : 4;
+    const size_t kes = src_host->k_kind == 1 ? 4 : 2;
     // Keys are streamed in full by the scoring kernel, so they are copied.  Values and positions are only read
     // for the kept rows: when the host arrays are device-accessible (pinned, mapped), the gather reads those
     // rows straight from host memory and the bulk copies are skipped.

@@ -60,6 +60,54 @@ def test_config0_tiny_fp32_pre_rope():
     assert torch.equal(kout[0, 0, 0], kpre[0, 0, 0][sel])
 
 
+@pytest.mark.parametrize("G,layout", [(4, 0), (8, 0), (3, 1)])
+def test_bf16_pre_rope_keys(G, layout):
+    """k_kind 2: the cache holds the pre-RoPE vectors k_f of Section 4.1 in bf16, each slot with its position (here
+    scattered, ascending, up to 60,000 below the query).  Scored in fp32 with tabulated distance phasors; against the
+    oracle's pre-RoPE reading on the same bf16 values, then selection and compaction as for any cache."""
+    N, B, H = 2500, 300, 2
+    sp = W.SPECS["tiny"].scaled(name=f"pre{G}{layout}", n_kv_heads=H, group_size=G, n_keys=N, budget=B)
+    w = W.make_workload(sp, DEV)
+    kpre = w.k_pre_fp32.to(torch.bfloat16)                                   # [1, 1, H, N, 128], interleaved pairs
+    g = torch.Generator().manual_seed(9)
+    pos = torch.stack([torch.sort(torch.randperm(50000, generator=g)[:N]).values for _ in range(H)]).to(torch.int32)
+    p_q = 60000
+    qc, qn = w.q_center, w.q_mean_norm
+    k_dev, qc_dev = kpre, qc
+    if layout == 1:
+        perm = torch.cat([torch.arange(0, 128, 2), torch.arange(1, 128, 2)])
+        k_dev, qc_dev = kpre[..., perm.to(DEV)].contiguous(), qc[..., perm].contiguous()
+    ctx = tb.TriContext(1, H, G, qc_dev, qn, rope_theta=sp.theta, pair_layout=layout)
+    positions = pos.view(1, 1, H, N).to(DEV)
+    cur = torch.tensor([p_q], dtype=torch.int64, device=DEV)
+    src = tb.CacheView(k_dev, w.v, seq_lens=w.seq_lens, positions=positions, pre_rope=True)
+    ws = ctx.workspace(1, N, B)
+    scores = torch.empty(H, N, dtype=torch.float32, device=DEV)
+    raw = torch.empty(H, N, G, dtype=torch.float32, device=DEV)
+    ctx.score(src, cur, scores, ws, raw=raw)
+    k2 = torch.zeros(1, 1, H, B, 128, dtype=torch.bfloat16, device=DEV); v2 = torch.zeros_like(k2)
+    p2 = torch.zeros(1, 1, H, B, dtype=torch.int32, device=DEV)
+    idx = torch.empty(H, B, dtype=torch.int32, device=DEV); cnt = torch.empty(H, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ctx.compress(src, cur, B, tb.CacheView(k2, v2, positions=p2, pre_rope=True), ws, kept_idx=idx, kept_cnt=cnt, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status) == 0
+    for h in range(H):
+        raw_o = oracle.score_raw(kpre[0, 0, h].double().cpu().numpy(), pos[h].numpy(), p_q, qc[0, h * G:(h + 1) * G].double().numpy(),
+                                 qn[0, h * G:(h + 1) * G].double().numpy(), theta=sp.theta)
+        _, s_o = oracle.normalize(raw_o)
+        ref = dict(raw=raw_o, s_final=s_o, idx=oracle.select(s_o, B), k=k_dev[0, 0, h].cpu(), v=w.v[0, 0, h].cpu(), pos=pos[h].long())
+        check_scores(raw[h].cpu().numpy(), scores[h].cpu().numpy(), ref)
+        got = idx[h].cpu().numpy()
+        check_kept(got, int(cnt[h]), ref, B)
+        check_compacted(k2[0, 0, h], v2[0, 0, h], p2[0, 0, h], got, ref)
+    # a distance outside the phasor tables is reported, not mis-scored silently
+    far = torch.tensor([p_q + (1 << 21)], dtype=torch.int64, device=DEV)
+    ctx.compress(src, far, B, tb.CacheView(k2, v2, positions=p2, pre_rope=True), ws, kept_idx=idx, kept_cnt=cnt, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status) == 5
+
+
 def test_config1_shape_scaled():
     """Qwen3-8B head geometry (G = 4), 2 layers x 2 KV heads, 5,000 keys: 3 scoring blocks + ragged tail."""
     sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(n_layers=2, n_kv_heads=2, n_keys=5000, budget=300)
