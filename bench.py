@@ -48,7 +48,7 @@ NOMINAL_HBM_GBS = 8000.0
 SCORE_TRAFFIC = {"bytes_per_key": (268499200 + 14236928) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
-                 "sha256": "09de78855e1affb1a48f05f07ba6eacd415f15845f53292a8431f791b9374d0e"}
+                 "sha256": "39c817c58bdfb35b2b941cd822f77c33e4c616877bb032589dcc0c0286a25f7b"}
 
 
 def score_traffic_per_launch(keys):

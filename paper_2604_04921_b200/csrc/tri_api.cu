@@ -13,6 +13,7 @@
 #include "tri_calib.cuh"
 #include "tri_compact.cuh"
 #include "tri_score.cuh"
+#include "tri_score_pre.cuh"
 #include "tri_score_tma.cuh"
 #include "tri_score_umma.cuh"
 #include "tri_select.cuh"

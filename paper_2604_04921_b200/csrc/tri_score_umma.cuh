@@ -17,7 +17,7 @@
 //                   publishes the accumulator (two accumulators alternate)
 //   compute warps   (one tile later, under the next tile's MMAs) tcgen05.ld their row's columns, add the two
 //                   halves, store the raw scores and keep sum / sum of squares per head.
-// Every mbarrier wait is bounded; a wait that runs out sets TRI_ERR_TIMEOUT in device_status, all roles fall
+// Every mbarrier wait is bounded and sleeps between polls; a wait that runs out sets TRI_ERR_TIMEOUT in device_status, all roles fall
 // through to the common exit, and the tensor memory is released there.
 #pragma once
 #include <cuda.h>
@@ -48,21 +48,20 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
 }
-// Bounded wait whose polls let the hardware park the thread for up to `kParkNs` before answering: few polls,
-// few issue slots, and still a hard limit (polls x park time) after which the caller gives up.
-constexpr uint32_t kParkNs = 20000, kParkPolls = 1u << 12;
+// Bounded wait that sleeps between polls: a warp waiting for another role of the block must not spend the
+// issue slots the other blocks of the SM compute with.  One poll at once, then `nap` nanoseconds of sleep before
+// each further poll; after kNapPolls polls the caller gives up.
+constexpr uint32_t kNapPolls = 1u << 20;
+#ifndef TRI_UMMA_NAP
+#define TRI_UMMA_NAP 64
+#endif
+template <uint32_t NAP = TRI_UMMA_NAP>
 __device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity)
 {
-    for (uint32_t i = 0; i < kParkPolls; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n.reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
-            "selp.u32 %0, 1, 0, p;\n}\n"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity), "r"(kParkNs)
-            : "memory");
-        if (ok) return true;
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < kNapPolls; ++i) {
+        if (NAP) __nanosleep(NAP);
+        if (mbar_try_wait(bar, parity)) return true;
     }
     return false;
 }
