@@ -315,9 +315,11 @@ tri_status tri_calib_finalize(const void *state, int32_t n_heads, int32_t pair_l
                               float *q_mean_norm, float *mrl, void *stream);
 
 /*
- * Self-test of the bounded wait the scoring kernel uses for its copy-engine barriers (the paper has no
- * counterpart): one warp waits on a barrier that nothing ever completes, gives up after a short poll limit,
- * writes TRI_ERR_TIMEOUT to *device_status (device int32) and returns normally.  The context stays usable.
+ * Self-test of the bounded waits the scoring kernels use for their copy-engine and tensor-core barriers (the paper has no
+ * counterpart): one warp waits on a barrier that nothing ever completes, once with the spinning wait of the mma.sync
+ * kernel and once with the sleeping wait of the tcgen05 kernel; each gives up after a short poll limit.  *device_status
+ * (device int32) ends as TRI_ERR_TIMEOUT if both ran out, as TRI_ERR_DEVICE_CHECK if a wait claimed success; the kernels
+ * return normally and the context stays usable.
  */
 tri_status tri_selftest_bounded_wait(int32_t *device_status, void *stream);
 

@@ -961,7 +961,8 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
 extern "C" tri_status tri_selftest_bounded_wait(int32_t *device_status, void *stream)
 {
     if (!device_status) return TRI_ERR_INVALID_ARG;
-    k_selftest_wait<<<1, 32, 0, (cudaStream_t)stream>>>(device_status);
+    k_selftest_wait<<<1, 32, 0, (cudaStream_t)stream>>>(device_status);      // the spinning wait of the mma.sync kernel
+    k_selftest_nap<<<1, 32, 0, (cudaStream_t)stream>>>(device_status);       // the sleeping wait of the tcgen05 kernel
     return check_launch("k_selftest_wait");
 }
 

@@ -56,10 +56,10 @@ constexpr uint32_t kNapPolls = 1u << 20;
 #define TRI_UMMA_NAP 64
 #endif
 template <uint32_t NAP = TRI_UMMA_NAP>
-__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_parked(uint32_t bar, uint32_t parity, uint32_t polls = kNapPolls)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < kNapPolls; ++i) {
+    for (uint32_t i = 0; i < polls; ++i) {
         if (NAP) __nanosleep(NAP);
         if (mbar_try_wait(bar, parity)) return true;
     }
@@ -427,6 +427,22 @@ k_score_umma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kUTmemCols) : "memory");
     }
+}
+
+// The sleeping wait on a barrier that nothing completes: it must run out.  Leaves *device_status alone if it does (the
+// spinning self-test before it has set TRI_ERR_TIMEOUT there) and overwrites it with TRI_ERR_DEVICE_CHECK if the wait
+// claims success.
+__global__ void k_selftest_nap(int32_t *device_status)
+{
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    __syncwarp();
+    const bool done = mbar_wait_parked(b, 0, 1u << 8);
+    if (done && threadIdx.x == 0) atomicExch(device_status, (int)TRI_ERR_DEVICE_CHECK);
 }
 
 }  // namespace tri
