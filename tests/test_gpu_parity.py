@@ -585,12 +585,12 @@ def test_compact_standalone_and_rerun_determinism():
     assert torch.equal(p2, a["pos_out"]) and lens.tolist() == [sp.budget]
 
 
-@pytest.mark.parametrize("pinned,budget", [(True, 700), (False, 700), (True, 2048)])
-def test_host_resident_cache_round(pinned, budget):
+@pytest.mark.parametrize("pinned,budget,G", [(True, 700, 4), (False, 700, 4), (True, 2048, 4), (True, 700, 8)])
+def test_host_resident_cache_round(pinned, budget, G):
     """tri_compress_host: K/V/positions in host memory in, compacted rows in host memory out; with pinned
     arrays and at most half of the rows kept, V and positions are never copied in bulk (the gather reads the
     kept rows from host memory)."""
-    sp = W.SPECS["qwen3_8b_steady_b64"].scaled(name="hostpath", n_layers=2, n_kv_heads=2, n_seqs=3, budget=budget)
+    sp = W.SPECS["qwen3_8b_steady_b64"].scaled(name="hostpath", n_layers=2, n_kv_heads=2, n_seqs=3, budget=budget, group_size=G)
     w = W.make_workload(sp, DEV)
     ref = run_compress(w, sp.budget, want_scores=False)
     L, S, H, B, N = 2, 3, 2, sp.budget, sp.n_keys
@@ -646,10 +646,11 @@ def test_pipelined_round_is_bit_identical(kind):
             assert torch.equal(ref[key], got[key]), (ranges, key)
 
 
-def test_round_replays_from_a_cuda_graph():
+@pytest.mark.parametrize("G", [4, 8])
+def test_round_replays_from_a_cuda_graph(G):
     """tri_compress only enqueues kernels on the given stream (no allocation, no synchronisation), so a decode
     loop can capture one round in a CUDA graph and replay it; the replay reads cur_pos from device memory."""
-    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="graph", n_layers=2, n_kv_heads=2, n_keys=6000, budget=500)
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="graph", n_layers=2, n_kv_heads=2, n_keys=6000, budget=500, group_size=G)
     w = W.make_workload(sp, DEV)
     direct = run_compress(w, sp.budget, want_scores=False)           # also the first call: one-time kernel set-up
     ctx = direct["ctx"]
