@@ -152,6 +152,19 @@ def test_config4_shape_ragged_paged(in_place):
         check_unit(w, res, ref, *u, sp.budget)
 
 
+@pytest.mark.parametrize("page_size,G", [(64, 4), (32, 8), (128, 8)])
+def test_other_page_sizes(page_size, G):
+    """Pages of 32, 64 and 128 tokens (any multiple of 16 is accepted), both scoring kernels' copy loops, in place."""
+    sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name=f"pg{page_size}", n_layers=1, n_kv_heads=2, n_seqs=3, n_keys=3000,
+                                                  n_keys_min=500, budget=400, page_size=page_size, group_size=G)
+    w = W.make_workload(sp, DEV)
+    refs = {u: oracle_unit(w, *u, sp.budget) for u in _all_units(w)}
+    res = run_compress(w, sp.budget, in_place=True)
+    assert int(res["status"].item()) == 0
+    for u, ref in refs.items():
+        check_unit(w, res, ref, *u, sp.budget)
+
+
 def test_token_major_page_layout():
     """Pages stored [layer][page][slot][head][128] (head stride 128, slot stride H * 128): the view's strides
     describe it, nothing else changes."""
