@@ -82,19 +82,41 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float upper, float lower)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(r) : "f"(upper), "f"(lower));
     return r;
 }
-// |(re0, im0)| and |(re1, im1)| as a packed bf16 pair `hi` (first magnitude in the lower half) and the bf16
-// pair `lo` of what the rounding left over: hi + lo carries each magnitude to ~2^-17.
-__device__ __forceinline__ void mag_pair(float re0, float im0, float re1, float im1, uint32_t &hi, uint32_t &lo)
+// Two band magnitudes straight from packed bf16 words, with the mixed-precision FMA of sm_100 (bf16 x bf16 + fp32 in
+// one instruction, the product exact): no unpacking of the operands.
+//   PAIRED = false: word a = (re, im) of one band, word b = (re, im) of another      -> |a|, |b|
+//   PAIRED = true : word a = real parts of two bands, word b = their imaginary parts -> |(a.lo, b.lo)|, |(a.hi, b.hi)|
+// Result: `hi` = the two magnitudes rounded to bf16 (first in the lower half), `lo` = the bf16 of what the rounding
+// left over (m - hi, again one mixed FMA each): hi + lo carries each magnitude to ~2^-17.
+#define TRI_MAG_PAIR_ASM(X0, Y0, X1, Y1)                                                   \
+    asm("{\n"                                                                             \
+        ".reg .b16 a0, a1, b0, b1, h0, h1, neg1;\n"                                       \
+        ".reg .f32 s0, s1, m0, m1, r0, r1;\n"                                             \
+        "mov.b32 {a0, a1}, %2;\n"                                                         \
+        "mov.b32 {b0, b1}, %3;\n"                                                         \
+        "mov.b16 neg1, 0xBF80;\n" /* -1.0 in bf16 */                                      \
+        "fma.rn.f32.bf16 s0, " X0 ", " X0 ", 0f00000000;\n"                               \
+        "fma.rn.f32.bf16 s1, " X1 ", " X1 ", 0f00000000;\n"                               \
+        "fma.rn.f32.bf16 s0, " Y0 ", " Y0 ", s0;\n"                                       \
+        "fma.rn.f32.bf16 s1, " Y1 ", " Y1 ", s1;\n"                                       \
+        "sqrt.approx.ftz.f32 m0, s0;\n"                                                   \
+        "sqrt.approx.ftz.f32 m1, s1;\n"                                                   \
+        "cvt.rn.bf16x2.f32 %0, m1, m0;\n"                                                 \
+        "mov.b32 {h0, h1}, %0;\n"                                                         \
+        "fma.rn.f32.bf16 r0, h0, neg1, m0;\n"                                             \
+        "fma.rn.f32.bf16 r1, h1, neg1, m1;\n"                                             \
+        "cvt.rn.bf16x2.f32 %1, r1, r0;\n"                                                 \
+        "}\n"                                                                             \
+        : "=&r"(hi), "=r"(lo)                                                             \
+        : "r"(a), "r"(b))
+
+template <bool PAIRED>
+__device__ __forceinline__ void mag_pair(uint32_t a, uint32_t b, uint32_t &hi, uint32_t &lo)
 {
-    uint64_t re = pack2(re0, re1), im = pack2(im0, im1);
-    float s0, s1;
-    unpack2(fma2(re, re, mul2(im, im)), s0, s1);
-    const float m0 = fast_sqrt(s0), m1 = fast_sqrt(s1);
-    hi = cvt_bf16x2(m1, m0);
-    float r0, r1;
-    unpack2(sub2(pack2(m0, m1), pack2(bf16_lo(hi), bf16_hi(hi))), r0, r1);
-    lo = cvt_bf16x2(r1, r0);
+    if (PAIRED) TRI_MAG_PAIR_ASM("a0", "b0", "a1", "b1");
+    else TRI_MAG_PAIR_ASM("a0", "a1", "b0", "b1");
 }
+#undef TRI_MAG_PAIR_ASM
 
 template <int NT, int LAYOUT>
 __global__ void __launch_bounds__(kScoreThreads, 3)
@@ -233,15 +255,15 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
             uint32_t hA[4], lA[4];
             if (LAYOUT == 0) {
                 const uint32_t *a = X[2 * pr], *b = X[2 * pr + 1];      // one register = (re, im) of one band
-                mag_pair(bf16_lo(a[0]), bf16_hi(a[0]), bf16_lo(a[2]), bf16_hi(a[2]), hA[0], lA[0]);
-                mag_pair(bf16_lo(a[1]), bf16_hi(a[1]), bf16_lo(a[3]), bf16_hi(a[3]), hA[1], lA[1]);
-                mag_pair(bf16_lo(b[0]), bf16_hi(b[0]), bf16_lo(b[2]), bf16_hi(b[2]), hA[2], lA[2]);
-                mag_pair(bf16_lo(b[1]), bf16_hi(b[1]), bf16_lo(b[3]), bf16_hi(b[3]), hA[3], lA[3]);
+                mag_pair<false>(a[0], a[2], hA[0], lA[0]);
+                mag_pair<false>(a[1], a[3], hA[1], lA[1]);
+                mag_pair<false>(b[0], b[2], hA[2], lA[2]);
+                mag_pair<false>(b[1], b[3], hA[3], lA[3]);
             } else {
                 const uint32_t *re = X[pr], *im = X[pr + 4];            // two bands per register, re and im apart
 #pragma unroll
                 for (int x = 0; x < 4; ++x)
-                    mag_pair(bf16_lo(re[x]), bf16_lo(im[x]), bf16_hi(re[x]), bf16_hi(im[x]), hA[x], lA[x]);
+                    mag_pair<true>(re[x], im[x], hA[x], lA[x]);
             }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {

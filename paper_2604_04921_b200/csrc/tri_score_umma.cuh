@@ -335,17 +335,17 @@ k_score_umma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
                     if (LAYOUT == 0) {               // block hs holds bands 32 hs .. 32 hs + 31; a register = (re, im) of one band
                         a = *reinterpret_cast<const uint4 *>(ka + hs * kUBlockBytes + sw128(row, 2 * i));
                         b = *reinterpret_cast<const uint4 *>(ka + hs * kUBlockBytes + sw128(row, 2 * i + 1));
-                        mag_pair(bf16_lo(a.x), bf16_hi(a.x), bf16_lo(a.y), bf16_hi(a.y), hi[0], lo[0]);
-                        mag_pair(bf16_lo(a.z), bf16_hi(a.z), bf16_lo(a.w), bf16_hi(a.w), hi[1], lo[1]);
-                        mag_pair(bf16_lo(b.x), bf16_hi(b.x), bf16_lo(b.y), bf16_hi(b.y), hi[2], lo[2]);
-                        mag_pair(bf16_lo(b.z), bf16_hi(b.z), bf16_lo(b.w), bf16_hi(b.w), hi[3], lo[3]);
+                        mag_pair<false>(a.x, a.y, hi[0], lo[0]);
+                        mag_pair<false>(a.z, a.w, hi[1], lo[1]);
+                        mag_pair<false>(b.x, b.y, hi[2], lo[2]);
+                        mag_pair<false>(b.z, b.w, hi[3], lo[3]);
                     } else {                         // a = real parts (block 0), b = imaginary parts (block 1), two bands per register
                         a = *reinterpret_cast<const uint4 *>(ka + sw128(row, 4 * hs + i));
                         b = *reinterpret_cast<const uint4 *>(ka + kUBlockBytes + sw128(row, 4 * hs + i));
-                        mag_pair(bf16_lo(a.x), bf16_lo(b.x), bf16_hi(a.x), bf16_hi(b.x), hi[0], lo[0]);
-                        mag_pair(bf16_lo(a.y), bf16_lo(b.y), bf16_hi(a.y), bf16_hi(b.y), hi[1], lo[1]);
-                        mag_pair(bf16_lo(a.z), bf16_lo(b.z), bf16_hi(a.z), bf16_hi(b.z), hi[2], lo[2]);
-                        mag_pair(bf16_lo(a.w), bf16_lo(b.w), bf16_hi(a.w), bf16_hi(b.w), hi[3], lo[3]);
+                        mag_pair<true>(a.x, b.x, hi[0], lo[0]);
+                        mag_pair<true>(a.y, b.y, hi[1], lo[1]);
+                        mag_pair<true>(a.z, b.z, hi[2], lo[2]);
+                        mag_pair<true>(a.w, b.w, hi[3], lo[3]);
                     }
                     tc_st4(mag + 4 * i, hi[0], hi[1], hi[2], hi[3]);
                     tc_st4(mag + 32 + 4 * i, lo[0], lo[1], lo[2], lo[3]);
