@@ -297,11 +297,13 @@ k_score_umma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
             if (!ok) { gave_up = 1; break; }
             tc_fence_after();
             if (lane == 0) {
+                // the key stage has served both its readers (the trigonometric MMAs issued above and the compute warps,
+                // whose arrival was just seen): it may be refilled as soon as those MMAs have completed
+                tc_commit(b_kempty + 8 * st);
                 const uint32_t mag = tmem + kUMagCol + mb * kUMagCols;
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     tc_mma_bf16_ts(acc, mag + 8 * k, tc_desc_sw128(sm_bn + (k >> 2) * (NCOL * 128) + (k & 3) * 32), idesc, 1u);
-                tc_commit(b_kempty + 8 * st);      // the key stage may be refilled
                 tc_commit(b_accfull + 8 * a);      // the accumulator may be read, the magnitude buffer rewritten
             }
             __syncwarp();
