@@ -265,7 +265,7 @@ def run_calibration(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "calibration qwen3_8b layer", "tokens": T, "heads": Hq, "storage_dtype": "bf16",
                        "l2": f"inputs larger than L2: {nbytes / 1e9:.2f} GB read per step"},
-            "roofline": {"kernel": "k_calib_partial (+ k_calib_merge)", "bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9,
+            "roofline": {"kernel": "k_calib_tma (+ k_calib_merge)", "bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9,
                          "peak": peak, "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / peak, "traffic": None,
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": nbytes},
             "gpu_launches": 2 * steps}

@@ -304,6 +304,10 @@ tri_status tri_profile_end(tri_ctx *ctx);
  *           multiples of 4 (q_kind 0: 8-byte rows) resp. 4 (q_kind 1: 16-byte rows); q aligned likewise
  *   ws      device scratch of tri_calib_workspace_bytes(n_heads, T) bytes, 8-byte aligned
  * Sums are formed in a fixed order (no atomics), so equal inputs give equal bits.
+ * Rows reach the SMs through the TMA unit when q is 16-byte aligned, both strides are multiples of 16 bytes and
+ * T < 2^31 (every contiguous tensor, every fp32 layout accepted here), through plain loads otherwise; the two paths
+ * cut the tokens into blocks alike and differ only in speed.  Every wait on a TMA copy is bounded: should one run
+ * out, the sums of the pass are set to NaN, so that tri_calib_finalize yields NaN instead of wrong means.
  */
 size_t     tri_calib_state_bytes(int32_t n_heads);
 size_t     tri_calib_workspace_bytes(int32_t n_heads, int64_t T);

@@ -20,7 +20,7 @@ _ROOT = _PKG.parent
 LIB_PATH = _PKG / "lib" / "libtriattn.so"
 SOURCES = [_PKG / "csrc" / "tri_api.cu"]
 HEADERS = [_ROOT / "include" / "tri_attention.h", _PKG / "csrc" / "tri_common.cuh", _PKG / "csrc" / "tri_score.cuh",
-           _PKG / "csrc" / "tri_score_pre.cuh", _PKG / "csrc" / "tri_score_tma.cuh", _PKG / "csrc" / "tri_score_umma.cuh", _PKG / "csrc" / "tri_calib.cuh",
+           _PKG / "csrc" / "tri_score_pre.cuh", _PKG / "csrc" / "tri_score_tma.cuh", _PKG / "csrc" / "tri_score_umma.cuh", _PKG / "csrc" / "tri_calib.cuh", _PKG / "csrc" / "tri_calib_tma.cuh",
            _PKG / "csrc" / "tri_select.cuh", _PKG / "csrc" / "tri_compact.cuh"]
 
 EXPORTS = ["tri_create", "tri_destroy", "tri_workspace_bytes", "tri_score", "tri_select", "tri_compact",

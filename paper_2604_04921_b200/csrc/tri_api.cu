@@ -11,6 +11,7 @@
 #include <nvtx3/nvToolsExt.h>
 
 #include "tri_calib.cuh"
+#include "tri_calib_tma.cuh"
 #include "tri_compact.cuh"
 #include "tri_score.cuh"
 #include "tri_score_pre.cuh"
@@ -336,7 +337,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, int32_t n_layers, CUtensorMap *out)
+tri_status encode_fn(EncodeTiledFn *out)
 {
     static EncodeTiledFn fn = nullptr;
     static std::mutex fn_mu;
@@ -348,6 +349,15 @@ tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, 
         if (e != cudaSuccess || !ptr) return cuda_fail(e == cudaSuccess ? cudaErrorUnknown : e, "cuTensorMapEncodeTiled lookup");
         fn = (EncodeTiledFn)ptr;
     }
+    *out = fn;
+    return TRI_OK;
+}
+
+tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, int32_t n_layers, CUtensorMap *out)
+{
+    EncodeTiledFn fn;
+    tri_status fs = encode_fn(&fn);
+    if (fs != TRI_OK) return fs;
     auto bytes = [](int64_t elems) { return (cuuint64_t)(elems > 0 ? elems : 8) * 2; };
     cuuint64_t dims[5], strides[4];
     dims[0] = kHeadDim;
@@ -1078,9 +1088,48 @@ void calib_shape(int32_t n_heads, int64_t T, int32_t *nblocks, int32_t *per_bloc
     int64_t nb = want < most ? want : most;
     if (nb > 1024) nb = 1024;
     if (nb < 1) nb = 1;
-    int64_t per = (T + nb - 1) / nb;
+    int64_t per = ((T + nb - 1) / nb + 15) / 16 * 16;      // whole 16-token tiles
     *per_block = (int32_t)per;
     *nblocks = (int32_t)((T + per - 1) / per);
+}
+
+// The queries as a rank-3 tensor (component, head, token) for the TMA unit, box = one 4 KB tile of one head.
+// false when the layout does not meet the unit's alignment rules (the caller then takes the plain-load kernel).
+bool calib_tma_ok(const void *q, int32_t q_kind, int64_t T, int32_t n_heads, int64_t stride_tok, int64_t stride_head)
+{
+    const int64_t es = q_kind == 0 ? 2 : 4;
+    if (((uintptr_t)q & 15) || (stride_tok * es) % 16 || stride_tok <= 0 || T >= (int64_t)1 << 31) return false;
+    if (n_heads > 1 && ((stride_head * es) % 16 || stride_head <= 0)) return false;
+    return stride_tok * es < ((int64_t)1 << 40) && stride_head * es < ((int64_t)1 << 40);
+}
+
+tri_status encode_calib_map(const void *q, int32_t q_kind, int64_t T, int32_t n_heads, int64_t stride_tok,
+                            int64_t stride_head, CUtensorMap *out)
+{
+    EncodeTiledFn fn;
+    tri_status fs = encode_fn(&fn);
+    if (fs != TRI_OK) return fs;
+    const cuuint64_t es = q_kind == 0 ? 2 : 4;
+    cuuint64_t dims[3] = {kHeadDim, (cuuint64_t)n_heads, (cuuint64_t)T};
+    cuuint64_t strides[2] = {(cuuint64_t)(n_heads > 1 ? stride_head : kHeadDim) * es, (cuuint64_t)stride_tok * es};
+    cuuint32_t box[3] = {kHeadDim, 1, (cuuint32_t)(kCalibTileBytes / (kHeadDim * es))}, estr[3] = {1, 1, 1};
+    CUresult r = fn(out, q_kind == 0 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                    const_cast<void *>(q), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_err, sizeof g_err, "cuTensorMapEncodeTiled (calibration) failed with CUresult %d", (int)r);
+        return TRI_ERR_CUDA;
+    }
+    return TRI_OK;
+}
+
+template <int LAYOUT, int KIND>
+tri_status launch_calib_tma(dim3 grid, cudaStream_t st, const CUtensorMap &map, const CalibParams &p)
+{
+    // the attribute belongs to (function, device): set it on the current device before every launch (cheap, no sync)
+    TRI_CUDA(cudaFuncSetAttribute(k_calib_tma<LAYOUT, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kCalibDynSmem));
+    k_calib_tma<LAYOUT, KIND><<<grid, kCalibThreads, kCalibDynSmem, st>>>(map, p);
+    return TRI_OK;
 }
 
 }  // namespace
@@ -1122,7 +1171,16 @@ extern "C" tri_status tri_calib_accumulate(const void *q, int32_t q_kind, int64_
     calib_shape(n_heads, T, &nb, &p.per_block);
     p.partials = (double *)ws;
     dim3 grid(nb, n_heads);
-    if (pair_layout == 0 && q_kind == 0) k_calib_partial<0, 0><<<grid, kCalibThreads, 0, st>>>(p);
+    if (calib_tma_ok(q, q_kind, T, n_heads, stride_tok, stride_head)) {
+        CUtensorMap map;
+        tri_status ms = encode_calib_map(q, q_kind, T, n_heads, stride_tok, stride_head, &map);
+        if (ms != TRI_OK) return ms;
+        if (pair_layout == 0 && q_kind == 0) ms = launch_calib_tma<0, 0>(grid, st, map, p);
+        else if (pair_layout == 0) ms = launch_calib_tma<0, 1>(grid, st, map, p);
+        else if (q_kind == 0) ms = launch_calib_tma<1, 0>(grid, st, map, p);
+        else ms = launch_calib_tma<1, 1>(grid, st, map, p);
+        if (ms != TRI_OK) return ms;
+    } else if (pair_layout == 0 && q_kind == 0) k_calib_partial<0, 0><<<grid, kCalibThreads, 0, st>>>(p);
     else if (pair_layout == 0) k_calib_partial<0, 1><<<grid, kCalibThreads, 0, st>>>(p);
     else if (q_kind == 0) k_calib_partial<1, 0><<<grid, kCalibThreads, 0, st>>>(p);
     else k_calib_partial<1, 1><<<grid, kCalibThreads, 0, st>>>(p);

@@ -38,6 +38,29 @@ def test_calibration_matches_oracle(dtype, layout):
     assert float(r.min()) >= 0.0 and float(r.max()) <= 1.0 + 1e-6
 
 
+@pytest.mark.parametrize("dtype,pitch,lead,tma", [(torch.bfloat16, 128, 0, True), (torch.bfloat16, 136, 8, True),
+                                                  (torch.bfloat16, 132, 4, False), (torch.float32, 132, 4, True)])
+def test_calibration_on_both_load_paths(dtype, pitch, lead, tma):
+    """Rows whose base and strides are multiples of 16 bytes are staged by the TMA unit (every fp32 layout the entry
+    point accepts is one); a bf16 view that starts 8 bytes into a wider buffer with a row pitch of 132 elements has
+    neither and takes the kernel on plain loads.  Both against the oracle, on enough tokens for several blocks per
+    head with a ragged last tile, and with a token stride that is not the head count times the row pitch."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="calib3", n_layers=1, n_kv_heads=1, group_size=3)
+    T, H = 40000 + 7, 3
+    q = W.make_queries(sp, 0, T, DEV, dtype=dtype)
+    wide = torch.zeros(T, H + 1, pitch, dtype=dtype, device=DEV)      # one spare head
+    view = wide[:, :H, lead:lead + 128]
+    view.copy_(q)
+    es = 2 if dtype == torch.bfloat16 else 4
+    assert (view.data_ptr() % 16 == 0 and view.stride(1) * es % 16 == 0 and view.stride(0) * es % 16 == 0) == tma
+    cal = tb.Calibrator(H)
+    cal.add(view)
+    qc, qn, r = cal.result()
+    torch.cuda.synchronize()
+    c_o, n_o, r_o = _oracle_all(q, 0)
+    _check(qc, c_o); _check(qn, n_o); _check(r, r_o)
+
+
 def test_calibration_streams_in_chunks_and_feeds_the_round():
     sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name="calib2", n_layers=1, n_kv_heads=2, n_keys=1500, budget=100)
     q = W.make_queries(sp, 0, 3 * W.N_CALIB + 17, DEV, dtype=torch.float32)
