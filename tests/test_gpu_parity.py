@@ -940,3 +940,39 @@ def test_full_size_config4_slab_sampled_units():
     for u, ref in refs.items():
         st = check_unit(w, res, ref, *u, sp.budget)
         assert "raw_err" in st
+
+
+@pytest.mark.parametrize("G,ties", [(4, False), (8, False), (3, False), (4, True)])
+def test_fused_selection_of_long_units_equals_the_two_step_path(G, ties):
+    """Units of at least 65,536 keys that keep at most an eighth take the one-sweep selection inside the fused round
+    (sampled lower bound of the threshold, listed keys, exact selection on the list, bitmap emit).  Its kept slots
+    must be the very ones tri_select finds in the final scores tri_score writes (the general three-sweep path, itself
+    bit-exact against the oracle), and the oracle's.  With ties = True every key row is a copy of one of 40 rows, so
+    a unit's scores take 40 values: the threshold falls inside a group of ~1,750 equal scores, the lowest slots of
+    the group must win, and the group's value bin overflows the in-kernel list, which sends the unit down the
+    general path from inside the one-sweep one."""
+    sp = W.SPECS["qwen3_8b_oneshot_32k"].scaled(name=f"long{G}{int(ties)}", n_layers=1, n_kv_heads=2, n_keys=70001, budget=1500,
+                                                group_size=G)
+    w = W.make_workload(sp, DEV)
+    if ties:
+        pick = torch.randint(0, 40, (sp.n_keys,), generator=torch.Generator().manual_seed(11)).to(DEV)
+        w.k.copy_(w.k[..., pick, :].clone())
+    res = run_compress(w, sp.budget)                       # fused round, then tri_score for the scores
+    assert int(res["status"].item()) == 0
+    ctx = res["ctx"]
+    U = 2
+    idx2 = torch.full((U, sp.budget), -1, dtype=torch.int32, device=DEV)
+    cnt2 = torch.zeros(U, dtype=torch.int32, device=DEV)
+    ctx.select(res["scores"], w.seq_lens, sp.n_keys, sp.budget, idx2, cnt2)
+    torch.cuda.synchronize()
+    assert torch.equal(cnt2, res["kept_cnt"].view(-1)) and torch.equal(idx2, res["kept_idx"].view(U, -1))
+    if ties:
+        sc = res["scores"].view(U, -1)
+        assert all(len(torch.unique(sc[u])) <= 40 for u in range(U))
+        kept = torch.gather(sc[0], 0, idx2[0].long())
+        t = kept.min()                                   # the threshold: some keys equal to it are kept, some are not
+        assert int((sc[0] == t).sum()) > int((kept == t).sum()) > 0
+        eq = torch.nonzero(sc[0] == t).view(-1)
+        assert torch.equal(idx2[0][kept == t].long(), eq[: int((kept == t).sum())])     # the lowest slots of the group
+    else:
+        check_unit(w, res, oracle_unit(w, 0, 0, 1, sp.budget), 0, 0, 1, sp.budget)
