@@ -44,11 +44,11 @@ NOMINAL_HBM_GBS = 8000.0
 
 
 # DRAM traffic of the scoring kernel from its ncu capture (dram__bytes_read.sum + dram__bytes_write.sum of one launch of
-# k_score_tma<1,0> on 1,048,576 keys: 268,499,200 B + 14,236,928 B), valid only for the kernel source it was taken on.
-SCORE_TRAFFIC = {"bytes_per_key": (268499200 + 14236928) / 1048576,
+# k_score_tma<1,0> on 1,048,576 keys: 268,527,872 B + 14,151,424 B), valid only for the kernel source it was taken on.
+SCORE_TRAFFIC = {"bytes_per_key": (268527872 + 14151424) / 1048576,
                  "sources": ["paper_2604_04921_b200/csrc/tri_score_tma.cuh", "paper_2604_04921_b200/csrc/tri_score.cuh",
                              "paper_2604_04921_b200/csrc/tri_common.cuh"],
-                 "sha256": "39c817c58bdfb35b2b941cd822f77c33e4c616877bb032589dcc0c0286a25f7b"}
+                 "sha256": "593d3dd118fbf9bc7c8d32a690de9d7e27d4efda005560991a4a4e1b577abc17"}
 
 
 def score_traffic_per_launch(keys):
