@@ -84,12 +84,18 @@ tri_status tri_destroy(tri_ctx *ctx);
  *                           row at  l*stride_layer + page*stride_page + h*stride_head + (n % page_size)*stride_slot
  */
 typedef struct {
-    void *k;                   /* keys: bf16 post-RoPE (k_kind 0), fp32 pre-RoPE (1) or bf16 pre-RoPE (2) */
-    void *v;                   /* values, bf16, same strides as k; NULL = no value cache        */
+    void *k;                   /* keys: bf16 post-RoPE (k_kind 0), fp32 pre-RoPE (1), bf16 pre-RoPE (2), e4m3 post-RoPE (3) */
+    void *v;                   /* values, bf16 (e4m3 with k_kind 3), same strides as k; NULL = no value cache */
     int32_t k_kind;            /* 0: bf16 as cached by the model (post-RoPE) -- the fast path
                                   1: fp32 pre-RoPE vectors, scored in double (a slow reference-style path)
                                   2: bf16 pre-RoPE vectors (the k_f of Section 4.1 as they are), scored in fp32 with
                                      tabulated distance phasors; p_q - p_k must lie in [0, 2^21)
+                                  3: 8-bit post-RoPE keys in e4m3 (4 exponent bits, bias 7, 3 mantissa bits, no
+                                     infinities), 128 bytes per row, values in the same format.  The paper has no
+                                     8-bit cache; a key counts as the value its byte encodes (a positive scale shared
+                                     by a unit's keys drops out of the z-score of Section 4.3).  Widened exactly to f16
+                                     in registers, then the same contractions on f16 tensor-core MMAs.  Strides are
+                                     multiples of 16 elements.  tri_compress_host does not take this format.
                                   1 and 2 need `positions`, or slot = position                                   */
     int32_t paged;
     int64_t stride_layer, stride_seq, stride_head, stride_tok;

@@ -61,6 +61,10 @@ def _load():
     lib.tri_oracle_unit_bf16.argtypes = [P, P, c_i64, c_i, c_i64, P, P, c_i, P, c_i, c_d, c_i, c_i,
                                          c_i64, P, P, P]
     lib.tri_oracle_unit_bf16.restype = c_i64
+    lib.tri_oracle_unit_e4m3.argtypes = lib.tri_oracle_unit_bf16.argtypes
+    lib.tri_oracle_unit_e4m3.restype = c_i64
+    lib.tri_oracle_e4m3_to_f64.argtypes = [P, c_i64, P]
+    lib.tri_oracle_e4m3_to_f64.restype = None
     lib.tri_oracle_calibrate.argtypes = [P, c_i64, c_i, c_i, P, P, P]
     lib.tri_oracle_calibrate.restype = None
     lib.tri_oracle_num_threads.argtypes = []
@@ -180,6 +184,33 @@ def unit_bf16(k_post_bits, pos, p_q: int, q_center, q_mean_norm, B: int, offsets
     s = np.empty(N, dtype=np.float64)
     idx = np.empty(max(min(N, int(B)), 0), dtype=np.int32)
     cnt = _load().tri_oracle_unit_bf16(_p(k_post_bits), _p(pos), N, d, int(p_q), _p(q_center),
+                                       _p(q_mean_norm), G, _p(offsets), offsets.size, float(theta),
+                                       int(layout), int(norm_variant), int(B), _p(raw), _p(s), _p(idx))
+    assert cnt == idx.size
+    return raw, s, idx
+
+
+def e4m3_to_f64(bits: np.ndarray) -> np.ndarray:
+    """e4m3 bit patterns (uint8) -> the values they encode."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().tri_oracle_e4m3_to_f64(_p(bits), bits.size, _p(out))
+    return out
+
+
+def unit_e4m3(k_post_bits, pos, p_q: int, q_center, q_mean_norm, B: int, offsets=DEFAULT_OFFSETS,
+              theta: float = 1e6, layout: int = 0, norm_variant: int = 0):
+    """unit_bf16 for a unit cached post-RoPE in e4m3 (given as uint8 bit patterns)."""
+    k_post_bits = np.ascontiguousarray(k_post_bits, dtype=np.uint8)
+    pos = _i64(pos)
+    q_center, q_mean_norm, offsets = _f64(q_center), _f64(q_mean_norm), _i64(offsets)
+    N, d = k_post_bits.shape
+    G = q_center.shape[0]
+    assert q_center.shape == (G, d) and q_mean_norm.shape == (G, d // 2) and pos.shape == (N,)
+    raw = np.empty((G, N), dtype=np.float64)
+    s = np.empty(N, dtype=np.float64)
+    idx = np.empty(max(min(N, int(B)), 0), dtype=np.int32)
+    cnt = _load().tri_oracle_unit_e4m3(_p(k_post_bits), _p(pos), N, d, int(p_q), _p(q_center),
                                        _p(q_mean_norm), G, _p(offsets), offsets.size, float(theta),
                                        int(layout), int(norm_variant), int(B), _p(raw), _p(s), _p(idx))
     assert cnt == idx.size

@@ -265,6 +265,51 @@ int64_t tri_oracle_unit_bf16(const uint16_t *k_post_bf16, const int64_t *pos, in
     return cnt;
 }
 
+/* ---- 8-bit caches ------------------------------------------------------------------ */
+
+/*
+ * The paper does not speak of 8-bit key caches; the reading taken here: a key stored as e4m3 stands for the value
+ * its eight bits encode, and everything of Sections 4.1-4.3 applies to that value unchanged (a positive scale shared
+ * by a unit's keys multiplies every raw score of the unit and drops out of the z-score).
+ * e4m3 (the 8-bit floating-point format with 4 exponent and 3 mantissa bits, bias 7, no infinities): bits s eeee mmm.
+ *   eeee = 0          : (-1)^s * 2^-6 * (mmm / 8)                (subnormal; +0 and -0)
+ *   eeee = 15, mmm = 7: not a number
+ *   otherwise         : (-1)^s * 2^(eeee - 7) * (1 + mmm / 8)    (largest finite value 448)
+ */
+void tri_oracle_e4m3_to_f64(const uint8_t *in, int64_t n, double *out)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        const int b = in[i], e = (b >> 3) & 15, m = b & 7;
+        double v;
+        if (e == 15 && m == 7) v = NAN;
+        else if (e == 0) v = ldexp((double)m / 8.0, -6);
+        else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+        out[i] = (b & 128) ? -v : v;
+    }
+}
+
+/* tri_oracle_unit_bf16 for a unit cached post-RoPE in e4m3: k_post_e4m3 [N][d] bytes. */
+int64_t tri_oracle_unit_e4m3(const uint8_t *k_post_e4m3, const int64_t *pos, int64_t N, int d,
+                             int64_t p_q, const double *q_center, const double *q_mean_norm,
+                             int G, const int64_t *offsets, int n_off, double theta, int layout,
+                             int norm_variant, int64_t B, double *raw, double *s_final,
+                             int32_t *kept_idx)
+{
+    double *k_post = (double *)malloc((size_t)N * d * sizeof(double));
+    double *k_pre = (double *)malloc((size_t)N * d * sizeof(double));
+    double *raw_l = raw ? raw : (double *)malloc((size_t)G * N * sizeof(double));
+    tri_oracle_e4m3_to_f64(k_post_e4m3, N * d, k_post);
+    tri_oracle_unrotate(k_post, pos, N, d, theta, layout, k_pre);
+    tri_oracle_score_raw(k_pre, pos, N, d, p_q, q_center, q_mean_norm, G, offsets, n_off, theta,
+                         layout, norm_variant, raw_l);
+    tri_oracle_normalize(raw_l, G, N, NULL, s_final);
+    int64_t cnt = tri_oracle_select(s_final, N, B, kept_idx);
+    if (!raw) free(raw_l);
+    free(k_post);
+    free(k_pre);
+    return cnt;
+}
+
 int tri_oracle_num_threads(void)
 {
 #ifdef _OPENMP

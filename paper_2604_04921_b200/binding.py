@@ -174,13 +174,15 @@ class CacheView:
     def c_view(self) -> _CacheView:
         k = self.k
         assert k.dim() == 5 and k.shape[-1] == 128 and k.stride(-1) == 1
+        fp8 = k.dtype == torch.float8_e4m3fn                 # e4m3 keys come with e4m3 values (k_kind 3)
         if self.v is not None:
-            assert self.v.shape == k.shape and self.v.stride() == k.stride() and self.v.dtype == torch.bfloat16
-        assert k.dtype in (torch.bfloat16, torch.float32)
+            assert self.v.shape == k.shape and self.v.stride() == k.stride()
+            assert self.v.dtype == (torch.float8_e4m3fn if fp8 else torch.bfloat16)
+        assert k.dtype in (torch.bfloat16, torch.float32, torch.float8_e4m3fn)
         cv = _CacheView()
         cv.k = k.data_ptr()
         cv.v = self.v.data_ptr() if self.v is not None else None
-        cv.k_kind = (2 if self.pre_rope else 0) if k.dtype == torch.bfloat16 else 1
+        cv.k_kind = 3 if fp8 else ((2 if self.pre_rope else 0) if k.dtype == torch.bfloat16 else 1)
         if self.page_table is None:
             cv.paged = 0
             cv.stride_layer, cv.stride_seq, cv.stride_head, cv.stride_tok = k.stride()[:4]

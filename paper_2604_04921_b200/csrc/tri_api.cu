@@ -306,20 +306,25 @@ View to_view(const tri_cache_view *v)
     return w;
 }
 
+// Bytes per key element / per value element of a view's format (fp8 caches hold V in fp8 too).
+int k_esize_of(int32_t k_kind) { return k_kind == 1 ? 4 : (k_kind == 3 ? 1 : 2); }
+int v_esize_of(int32_t k_kind) { return k_kind == 3 ? 1 : 2; }
+
 tri_status check_view(const tri_cache_view *v, bool need_lens)
 {
     if (!v || !v->k) return TRI_ERR_INVALID_ARG;
-    if (v->k_kind < 0 || v->k_kind > 2 || v->n_max <= 0) return TRI_ERR_INVALID_ARG;
+    if (v->k_kind < 0 || v->k_kind > 3 || v->n_max <= 0) return TRI_ERR_INVALID_ARG;
     if (need_lens && !v->seq_lens) return TRI_ERR_INVALID_ARG;
     if (((uintptr_t)v->k & 15) || ((uintptr_t)v->v & 15)) return TRI_ERR_INVALID_ARG;
-    if (v->stride_layer % 8 || v->stride_head % 8) return TRI_ERR_INVALID_ARG;
+    const int q = v->k_kind == 3 ? 16 : 8;            // strides in elements; every row starts on a 16-byte boundary
+    if (v->stride_layer % q || v->stride_head % q) return TRI_ERR_INVALID_ARG;
     if (v->paged) {
         if (!v->page_table || v->max_pages_per_seq <= 0 || v->page_size <= 0) return TRI_ERR_INVALID_ARG;
         if (v->page_size % kTileKeys) return TRI_ERR_UNSUPPORTED;
-        if (v->stride_page % 8 || v->stride_slot % 8 || v->stride_slot < kHeadDim) return TRI_ERR_INVALID_ARG;
+        if (v->stride_page % q || v->stride_slot % q || v->stride_slot < kHeadDim) return TRI_ERR_INVALID_ARG;
         if ((int64_t)v->max_pages_per_seq * v->page_size < v->n_max) return TRI_ERR_INVALID_ARG;
     } else {
-        if (v->stride_seq % 8 || v->stride_tok % 8 || v->stride_tok < kHeadDim) return TRI_ERR_INVALID_ARG;
+        if (v->stride_seq % q || v->stride_tok % q || v->stride_tok < kHeadDim) return TRI_ERR_INVALID_ARG;
     }
     return TRI_OK;
 }
@@ -358,7 +363,8 @@ tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, 
     EncodeTiledFn fn;
     tri_status fs = encode_fn(&fn);
     if (fs != TRI_OK) return fs;
-    auto bytes = [](int64_t elems) { return (cuuint64_t)(elems > 0 ? elems : 8) * 2; };
+    const bool key8 = v->k_kind == 3;               // e4m3 rows: 128 one-byte elements, one box per 16-row tile
+    auto bytes = [key8](int64_t elems) { return (cuuint64_t)(elems > 0 ? elems : 16) * (key8 ? 1 : 2); };
     cuuint64_t dims[5], strides[4];
     dims[0] = kHeadDim;
     dims[2] = (cuuint64_t)c->desc.n_kv_heads;
@@ -376,8 +382,8 @@ tri_status encode_key_map(const tri_ctx *c, const tri_cache_view *v, int32_t S, 
     }
     strides[1] = bytes(v->stride_head);
     strides[3] = bytes(v->stride_layer);
-    cuuint32_t box[5] = {kHeadDim / 2, kTileKeys, 1, 1, 1}, estr[5] = {1, 1, 1, 1, 1};
-    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, v->k, dims, strides, box, estr,
+    cuuint32_t box[5] = {(cuuint32_t)(key8 ? kHeadDim : kHeadDim / 2), kTileKeys, 1, 1, 1}, estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(out, key8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, v->k, dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -433,6 +439,14 @@ tri_status launch_score_tma_one(dim3 grid, cudaStream_t st, const CUtensorMap &m
 {
     k_score_tma<NT, LAYOUT><<<grid, kScoreThreads, kScoreDynSmem, st>>>(map, sp);
     return TRI_OK;
+}
+
+template <int LAYOUT>
+void launch_score_fp8(int NT, dim3 grid, cudaStream_t st, const CUtensorMap &map, const ScoreParams &sp)
+{
+    if (NT == 1) k_score_tma<1, LAYOUT, true><<<grid, kScoreThreads, kScoreDynSmem / 2, st>>>(map, sp);
+    else if (NT == 2) k_score_tma<2, LAYOUT, true><<<grid, kScoreThreads, kScoreDynSmem / 2, st>>>(map, sp);
+    else k_score_tma<4, LAYOUT, true><<<grid, kScoreThreads, kScoreDynSmem / 2, st>>>(map, sp);
 }
 
 template <int LAYOUT>
@@ -503,7 +517,14 @@ tri_status run_score(tri_ctx *c, const tri_cache_view *src, int32_t S, const int
     sp.raw = raw; sp.partials = part; sp.device_status = device_status;
     dim3 grid((unsigned)((size_t)un.count * pl.nchunks));
     int pr = prof_open(c, 1, st);
-    if (src->k_kind == 0) {
+    if (src->k_kind == 3) {
+        // e4m3 keys: the mma.sync kernel on f16 operands, whatever the setting for bf16 keys is
+        const int NT = G <= 4 ? 1 : (G <= 8 ? 2 : 4);
+        CUtensorMap map;
+        if ((r = encode_key_map(c, src, S, ly.count, &map)) != TRI_OK) return r;
+        if (c->desc.pair_layout == 0) launch_score_fp8<0>(NT, grid, st, map, sp);
+        else launch_score_fp8<1>(NT, grid, st, map, sp);
+    } else if (src->k_kind == 0) {
         int NT = G <= 4 ? 1 : (G <= 8 ? 2 : 4);
         CUtensorMap map;
         if ((r = encode_key_map(c, src, S, ly.count, &map)) != TRI_OK) return r;
@@ -584,7 +605,7 @@ bool aliases(const tri_cache_view *a, const tri_cache_view *b)
 // Whether the round compacts bf16 K + V in place: then the gather is two launches (tiled prefix, parallel pass).
 bool two_pass_compaction(const tri_cache_view *src, const tri_cache_view *dst)
 {
-    return aliases(src, dst) && src->k_kind != 1 && src->v && dst->v;
+    return aliases(src, dst) && (src->k_kind == 0 || src->k_kind == 2) && src->v && dst->v;
 }
 
 tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx, const int32_t *kept_cnt,
@@ -595,11 +616,12 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
     p.src = to_view(src); p.dst = to_view(dst);
     p.kept_idx = kept_idx; p.kept_cnt = kept_cnt; p.new_seq_lens = new_seq_lens;
     p.S = S; p.H = c->desc.n_kv_heads; p.budget = budget; p.u0 = un.first;
-    p.k_esize = src->k_kind == 1 ? 4 : 2;
+    p.k_esize = k_esize_of(src->k_kind);
+    p.v_esize = v_esize_of(src->k_kind);
     p.k_vec = kHeadDim * p.k_esize / 16;
-    p.v_vec = (src->v && dst->v) ? kHeadDim * 2 / 16 : 0;
+    p.v_vec = (src->v && dst->v) ? kHeadDim * p.v_esize / 16 : 0;
     p.device_status = device_status;
-    const bool rows16 = src->k_kind != 1 && p.v_vec != 0;     // bf16 K and V: the row-gather kernel applies
+    const bool rows16 = (src->k_kind == 0 || src->k_kind == 2) && p.v_vec != 0;     // bf16 K and V: the row-gather kernel applies
     const int U = un.count;
     dim3 grid(U, (budget + kFastRowsPerBlock - 1) / kFastRowsPerBlock);
     const int pr = prof_open(c, 4, st);
@@ -890,6 +912,7 @@ extern "C" tri_status tri_compress_host(tri_ctx *c, const tri_cache_view *src_ho
     if ((r = check_common(c, S, src_dev->n_max, budget)) != TRI_OK) return r;
     if (dst_dev->n_max < budget && dst_dev->n_max < src_dev->n_max) return TRI_ERR_INVALID_ARG;
     if (src_dev->k_kind != dst_dev->k_kind || !ws || ((uintptr_t)ws & 255)) return TRI_ERR_INVALID_ARG;
+    if (src_dev->k_kind == 3) return TRI_ERR_UNSUPPORTED;       // host-resident fp8 caches: not built
     cudaStream_t st = (cudaStream_t)stream;
     const int L = c->desc.n_layers, H = c->desc.n_kv_heads;
     const size_t kes = src_host->k_kind == 1 ? 4 : 2;

@@ -17,9 +17,10 @@ struct CompactParams {
     int32_t *new_seq_lens;     // [S] or NULL
     int32_t S, H, budget;
     int32_t u0;                // first unit of this launch
-    int32_t k_vec;             // 16-byte vectors per K row (16 for bf16, 32 for fp32)
-    int32_t v_vec;             // 16-byte vectors per V row (16, or 0 without a value cache)
+    int32_t k_vec;             // 16-byte vectors per K row (16 for bf16, 32 for fp32, 8 for fp8)
+    int32_t v_vec;             // 16-byte vectors per V row (16, 8 for fp8, or 0 without a value cache)
     int32_t k_esize;           // bytes per K element
+    int32_t v_esize;           // bytes per V element
     int32_t *device_status;
 };
 
@@ -146,7 +147,7 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather_any(const CompactPara
         const bool is_k = c < p.k_vec;
         const char *sb = is_k ? p.src.k : p.src.v;
         char *db = is_k ? p.dst.k : p.dst.v;
-        const int esz = is_k ? p.k_esize : 2;
+        const int esz = is_k ? p.k_esize : p.v_esize;
         const int cb = (is_k ? c : c - p.k_vec) * 16;
         uint4 val[kGatherRowsPerWarp];
         int64_t doff[kGatherRowsPerWarp];
@@ -274,7 +275,7 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace_any(const C
             if (so == -1 && c == 0 && p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
             if (so < 0) continue;
             stage[i] = c < p.k_vec ? ld_stream(p.src.k + so * p.k_esize + c * 16)
-                                   : ld_stream(p.src.v + so * 2 + (c - p.k_vec) * 16);
+                                   : ld_stream(p.src.v + so * p.v_esize + (c - p.k_vec) * 16);
         }
         if (p.dst.positions && threadIdx.x < rows) {
             const int srow = __ldg(idx + j0 + threadIdx.x);
@@ -289,7 +290,7 @@ __global__ void __launch_bounds__(kInplaceThreads) k_compact_inplace_any(const C
             const bool is_k = c < p.k_vec;
             if (dof < 0) { if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK); }
             else if (is_k) *reinterpret_cast<uint4 *>(p.dst.k + dof * p.k_esize + c * 16) = stage[i];
-            else *reinterpret_cast<uint4 *>(p.dst.v + dof * 2 + (c - p.k_vec) * 16) = stage[i];
+            else *reinterpret_cast<uint4 *>(p.dst.v + dof * p.v_esize + (c - p.k_vec) * 16) = stage[i];
         }
         if (p.dst.positions && threadIdx.x < rows && pos_s[threadIdx.x] >= 0 &&
             __ldg(idx + j0 + threadIdx.x) != j0 + (int)threadIdx.x)

@@ -88,40 +88,79 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float upper, float lower)
 //   PAIRED = true : word a = real parts of two bands, word b = their imaginary parts -> |(a.lo, b.lo)|, |(a.hi, b.hi)|
 // Result: `hi` = the two magnitudes rounded to bf16 (first in the lower half), `lo` = the bf16 of what the rounding
 // left over (m - hi, again one mixed FMA each): hi + lo carries each magnitude to ~2^-17.
-#define TRI_MAG_PAIR_ASM(X0, Y0, X1, Y1)                                                   \
+#define TRI_MAG_PAIR_ASM(T, NEG1, X0, Y0, X1, Y1)                                         \
     asm("{\n"                                                                             \
         ".reg .b16 a0, a1, b0, b1, h0, h1, neg1;\n"                                       \
         ".reg .f32 s0, s1, m0, m1, r0, r1;\n"                                             \
         "mov.b32 {a0, a1}, %2;\n"                                                         \
         "mov.b32 {b0, b1}, %3;\n"                                                         \
-        "mov.b16 neg1, 0xBF80;\n" /* -1.0 in bf16 */                                      \
-        "fma.rn.f32.bf16 s0, " X0 ", " X0 ", 0f00000000;\n"                               \
-        "fma.rn.f32.bf16 s1, " X1 ", " X1 ", 0f00000000;\n"                               \
-        "fma.rn.f32.bf16 s0, " Y0 ", " Y0 ", s0;\n"                                       \
-        "fma.rn.f32.bf16 s1, " Y1 ", " Y1 ", s1;\n"                                       \
+        "mov.b16 neg1, " NEG1 ";\n" /* -1.0 */                                            \
+        "fma.rn.f32." T " s0, " X0 ", " X0 ", 0f00000000;\n"                              \
+        "fma.rn.f32." T " s1, " X1 ", " X1 ", 0f00000000;\n"                              \
+        "fma.rn.f32." T " s0, " Y0 ", " Y0 ", s0;\n"                                      \
+        "fma.rn.f32." T " s1, " Y1 ", " Y1 ", s1;\n"                                      \
         "sqrt.approx.ftz.f32 m0, s0;\n"                                                   \
         "sqrt.approx.ftz.f32 m1, s1;\n"                                                   \
-        "cvt.rn.bf16x2.f32 %0, m1, m0;\n"                                                 \
+        "cvt.rn." T "x2.f32 %0, m1, m0;\n"                                                \
         "mov.b32 {h0, h1}, %0;\n"                                                         \
-        "fma.rn.f32.bf16 r0, h0, neg1, m0;\n"                                             \
-        "fma.rn.f32.bf16 r1, h1, neg1, m1;\n"                                             \
-        "cvt.rn.bf16x2.f32 %1, r1, r0;\n"                                                 \
+        "fma.rn.f32." T " r0, h0, neg1, m0;\n"                                            \
+        "fma.rn.f32." T " r1, h1, neg1, m1;\n"                                            \
+        "cvt.rn." T "x2.f32 %1, r1, r0;\n"                                                \
         "}\n"                                                                             \
         : "=&r"(hi), "=r"(lo)                                                             \
         : "r"(a), "r"(b))
 
-template <bool PAIRED>
+// F16 = false: the words hold bf16 pairs and so do the results; true: f16 (the 8-bit key path widens its keys to f16).
+template <bool PAIRED, bool F16 = false>
 __device__ __forceinline__ void mag_pair(uint32_t a, uint32_t b, uint32_t &hi, uint32_t &lo)
 {
-    if (PAIRED) TRI_MAG_PAIR_ASM("a0", "b0", "a1", "b1");
-    else TRI_MAG_PAIR_ASM("a0", "a1", "b0", "b1");
+    if (F16) {
+        if (PAIRED) TRI_MAG_PAIR_ASM("f16", "0xBC00", "a0", "b0", "a1", "b1");
+        else TRI_MAG_PAIR_ASM("f16", "0xBC00", "a0", "a1", "b0", "b1");
+    } else {
+        if (PAIRED) TRI_MAG_PAIR_ASM("bf16", "0xBF80", "a0", "b0", "a1", "b1");
+        else TRI_MAG_PAIR_ASM("bf16", "0xBF80", "a0", "a1", "b0", "b1");
+    }
 }
 #undef TRI_MAG_PAIR_ASM
 
-template <int NT, int LAYOUT>
+// ---- 8-bit keys (e4m3): widened exactly to f16 in registers, then the same two contractions on f16 tensor-core MMAs ----
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// The two e4m3 values in the lower (upper) half of w as an f16 pair; every e4m3 value is an f16 value.
+__device__ __forceinline__ void e4m3x4_to_f16x2(uint32_t w, uint32_t &lo, uint32_t &hi)
+{
+    asm("{\n.reg .b16 a, b;\nmov.b32 {a, b}, %2;\ncvt.rn.f16x2.e4m3x2 %0, a;\ncvt.rn.f16x2.e4m3x2 %1, b;\n}\n"
+        : "=r"(lo), "=r"(hi) : "r"(w));
+}
+__device__ __forceinline__ uint32_t f16_bits(float w)          // f16(w), round to nearest even
+{
+    uint16_t r;
+    asm("cvt.rn.f16.f32 %0, %1;\n" : "=h"(r) : "f"(w));
+    return r;
+}
+__device__ __forceinline__ float f16_value(uint32_t bits)
+{
+    float r;
+    asm("cvt.f32.f16 %0, %1;\n" : "=f"(r) : "h"((uint16_t)bits));
+    return r;
+}
+
+// KEY8 = false: bf16 keys, tiles of two 64-element halves.  KEY8 = true: e4m3 keys, 128-byte rows, one box per tile;
+// a 32-bit register of the 8-bit fragment holds dims 4t .. 4t+3 of its k-step, so slot x of lane t stands for dim
+// 4t + x (not 2t + (x & 1) + 8 (x >> 1)): the B fragments are folded in the same order and the sum over k is the same.
+template <int NT, int LAYOUT, bool KEY8 = false>
 __global__ void __launch_bounds__(kScoreThreads, 3)
 k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
 {
+    constexpr int kTileB = KEY8 ? kTileBytes / 2 : kTileBytes;          // bytes of one 16-key tile
     extern __shared__ __align__(1024) uint8_t tiles[];   // [warp][stage][half][16 rows][128 B]
     __shared__ uint2 trigB[NT][8][32];
     __shared__ uint2 normB[NT][4][32];
@@ -139,7 +178,7 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
     const int ntiles = (key_end - key_begin + kTileKeys - 1) / kTileKeys;
     const int my_n = warp < ntiles ? (ntiles - warp + kScoreWarps - 1) / kScoreWarps : 0;
 
-    const uint32_t my_tiles = smem_u32(tiles) + warp * (kStages * kTileBytes);
+    const uint32_t my_tiles = smem_u32(tiles) + warp * (kStages * kTileB);
     const uint32_t my_bars = smem_u32(&bars[warp][0]);
 
     // lane 0 of each warp arms stage `it % kStages` with tile `it` of this warp
@@ -157,10 +196,10 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
             c1 = row - pg * p.src.page_size;
             c3 = page;
         }
-        const uint32_t bar = my_bars + stage * 8, dst = my_tiles + stage * kTileBytes;
-        mbar_expect_tx(bar, kTileBytes);
+        const uint32_t bar = my_bars + stage * 8, dst = my_tiles + stage * kTileB;
+        mbar_expect_tx(bar, kTileB);
         tma_load_5d(dst, &tmap, bar, 0, c1, h, c3, l);
-        tma_load_5d(dst + kTileBytes / 2, &tmap, bar, kHeadDim / 2, c1, h, c3, l);
+        if (!KEY8) tma_load_5d(dst + kTileBytes / 2, &tmap, bar, kHeadDim / 2, c1, h, c3, l);
     };
 
     if (lane == 0) {
@@ -181,15 +220,20 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
         if (g < G) {
 #pragma unroll
             for (int x = 0; x < 4; ++x) {            // k slots 2t, 2t+1, 2t+8, 2t+9 of step st = dims of the key row
-                const int d = 16 * st + 2 * t + (x & 1) + 8 * (x >> 1);
+                const int d = KEY8 ? 16 * st + 4 * t + x : 16 * st + 2 * t + (x & 1) + 8 * (x >> 1);
                 const int f = LAYOUT == 0 ? d >> 1 : d & (kBands - 1);
                 const bool imag = LAYOUT == 0 ? (d & 1) : (d >= kBands);
                 const int ir = LAYOUT == 0 ? 2 * f : f, ii = LAYOUT == 0 ? 2 * f + 1 : f + kBands;
                 const double cr = c[ir], ci = c[ii];
                 const double2 e = p.E[s * kBands + f];
                 const float v = imag ? (float)(cr * e.y + ci * e.x) : (float)(cr * e.x - ci * e.y);
-                const uint32_t hi = bf16_hi_bits(v);
-                w[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+                if (KEY8) {
+                    const uint32_t hi = f16_bits(v);
+                    w[x] = part == 0 ? hi : f16_bits(v - f16_value(hi));
+                } else {
+                    const uint32_t hi = bf16_hi_bits(v);
+                    w[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+                }
             }
         }
         trigB[nt][st][ln] = make_uint2(w[0] | (w[1] << 16), w[2] | (w[3] << 16));
@@ -197,15 +241,22 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
         // stand for the bands whose magnitudes the main loop puts there
         if (st < 4) {
             int bnd[4];
-            if (LAYOUT == 0) { bnd[0] = 16 * st + t; bnd[1] = 16 * st + 4 + t; bnd[2] = 16 * st + 8 + t; bnd[3] = 16 * st + 12 + t; }
+            if (KEY8 && LAYOUT == 0) { bnd[0] = 16 * st + 2 * t; bnd[1] = bnd[0] + 1; bnd[2] = 16 * st + 8 + 2 * t; bnd[3] = bnd[2] + 1; }
+            else if (KEY8) { bnd[0] = 16 * st + 4 * t; bnd[1] = bnd[0] + 1; bnd[2] = bnd[0] + 2; bnd[3] = bnd[0] + 3; }
+            else if (LAYOUT == 0) { bnd[0] = 16 * st + t; bnd[1] = 16 * st + 4 + t; bnd[2] = 16 * st + 8 + t; bnd[3] = 16 * st + 12 + t; }
             else { bnd[0] = 16 * st + 2 * t; bnd[1] = bnd[0] + 1; bnd[2] = 16 * st + 8 + 2 * t; bnd[3] = bnd[2] + 1; }
             uint32_t m[4] = {0u, 0u, 0u, 0u};
             if (g < G) {
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
                     const float v = p.mw[qh * kBands + bnd[x]];
-                    const uint32_t hi = bf16_hi_bits(v);
-                    m[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+                    if (KEY8) {
+                        const uint32_t hi = f16_bits(v);
+                        m[x] = part == 0 ? hi : f16_bits(v - f16_value(hi));
+                    } else {
+                        const uint32_t hi = bf16_hi_bits(v);
+                        m[x] = part == 0 ? hi : bf16_hi_bits(v - __uint_as_float(hi << 16));
+                    }
                 }
             }
             normB[nt][st][ln] = make_uint2(m[0] | (m[1] << 16), m[2] | (m[3] << 16));
@@ -225,13 +276,28 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
 
     for (int it = 0; it < my_n; ++it) {
         const int stage = it % kStages;
-        const uint32_t bar = my_bars + stage * 8, base = my_tiles + stage * kTileBytes;
+        const uint32_t bar = my_bars + stage * 8, base = my_tiles + stage * kTileB;
         if (!mbar_wait_bounded(bar, (it / kStages) & 1)) { timed_out = true; break; }
         uint32_t X[8][4];
+        if (KEY8) {
+            // one ldmatrix.x4 per 32 dims: registers = (row q | row q+8) x (dims 4t..4t+3 | 16+4t..16+4t+3) of the step;
+            // each widens to the A fragments of two f16 MMAs (slots: dims 4t, 4t+1 | row+8 | dims 4t+2, 4t+3 | row+8)
 #pragma unroll
-        for (int st = 0; st < 8; ++st) {
-            const int c = 2 * (st & 3) + lsel;
-            ldmatrix_x4(X[st], base + (st >> 2) * (kTileBytes / 2) + lrow * 128 + ((c ^ (lrow & 7)) << 4));
+            for (int s32 = 0; s32 < 4; ++s32) {
+                uint32_t r[4];
+                const int c = 2 * s32 + lsel;
+                ldmatrix_x4(r, base + lrow * 128 + ((c ^ (lrow & 7)) << 4));
+                e4m3x4_to_f16x2(r[0], X[2 * s32][0], X[2 * s32][2]);
+                e4m3x4_to_f16x2(r[1], X[2 * s32][1], X[2 * s32][3]);
+                e4m3x4_to_f16x2(r[2], X[2 * s32 + 1][0], X[2 * s32 + 1][2]);
+                e4m3x4_to_f16x2(r[3], X[2 * s32 + 1][1], X[2 * s32 + 1][3]);
+            }
+        } else {
+#pragma unroll
+            for (int st = 0; st < 8; ++st) {
+                const int c = 2 * (st & 3) + lsel;
+                ldmatrix_x4(X[st], base + (st >> 2) * (kTileBytes / 2) + lrow * 128 + ((c ^ (lrow & 7)) << 4));
+            }
         }
         __syncwarp();
         if (lane == 0 && it + kStages < my_n) {
@@ -247,7 +313,8 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 uint2 b = trigB[nt][st][lane];
-                mma_bf16_16816(acc[nt], X[st][0], X[st][1], X[st][2], X[st][3], b.x, b.y);
+                if (KEY8) mma_f16_16816(acc[nt], X[st][0], X[st][1], X[st][2], X[st][3], b.x, b.y);
+                else mma_bf16_16816(acc[nt], X[st][0], X[st][1], X[st][2], X[st][3], b.x, b.y);
             }
         }
 #pragma unroll
@@ -255,21 +322,26 @@ k_score_tma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
             uint32_t hA[4], lA[4];
             if (LAYOUT == 0) {
                 const uint32_t *a = X[2 * pr], *b = X[2 * pr + 1];      // one register = (re, im) of one band
-                mag_pair<false>(a[0], a[2], hA[0], lA[0]);
-                mag_pair<false>(a[1], a[3], hA[1], lA[1]);
-                mag_pair<false>(b[0], b[2], hA[2], lA[2]);
-                mag_pair<false>(b[1], b[3], hA[3], lA[3]);
+                mag_pair<false, KEY8>(a[0], a[2], hA[0], lA[0]);
+                mag_pair<false, KEY8>(a[1], a[3], hA[1], lA[1]);
+                mag_pair<false, KEY8>(b[0], b[2], hA[2], lA[2]);
+                mag_pair<false, KEY8>(b[1], b[3], hA[3], lA[3]);
             } else {
                 const uint32_t *re = X[pr], *im = X[pr + 4];            // two bands per register, re and im apart
 #pragma unroll
                 for (int x = 0; x < 4; ++x)
-                    mag_pair<true>(re[x], im[x], hA[x], lA[x]);
+                    mag_pair<true, KEY8>(re[x], im[x], hA[x], lA[x]);
             }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const uint2 b = normB[nt][pr][lane];
-                mma_bf16_16816(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
-                mma_bf16_16816(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
+                if (KEY8) {
+                    mma_f16_16816(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
+                    mma_f16_16816(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
+                } else {
+                    mma_bf16_16816(acc[nt], hA[0], hA[1], hA[2], hA[3], b.x, b.y);
+                    mma_bf16_16816(acc[nt], lA[0], lA[1], lA[2], lA[3], b.x, b.y);
+                }
             }
         }
 

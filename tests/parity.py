@@ -41,9 +41,13 @@ def oracle_unit(w: W.Workload, l: int, s: int, h: int, budget: int, offsets=orac
     G = w.spec.group_size
     qc = w.q_center[l, h * G:(h + 1) * G].double().numpy()
     qn = w.q_mean_norm[l, h * G:(h + 1) * G].double().numpy()
-    raw, sfin, idx = oracle.unit_bf16(W.bf16_bits(kk), pos.numpy(), int(w.cur_pos[s].item()), qc, qn, budget,
-                                      offsets=offsets, theta=w.spec.theta, layout=layout,
-                                      norm_variant=norm_variant)
+    if kk.dtype == torch.float8_e4m3fn:
+        raw, sfin, idx = oracle.unit_e4m3(kk.contiguous().view(torch.uint8).numpy(), pos.numpy(), int(w.cur_pos[s].item()), qc, qn,
+                                          budget, offsets=offsets, theta=w.spec.theta, layout=layout, norm_variant=norm_variant)
+    else:
+        raw, sfin, idx = oracle.unit_bf16(W.bf16_bits(kk), pos.numpy(), int(w.cur_pos[s].item()), qc, qn, budget,
+                                          offsets=offsets, theta=w.spec.theta, layout=layout,
+                                          norm_variant=norm_variant)
     return dict(raw=raw, s_final=sfin, idx=idx, k=kk, v=vv, pos=pos)
 
 
@@ -81,9 +85,10 @@ def check_compacted(k_out, v_out, pos_out, idx_gpu: np.ndarray, ref: dict):
     """Rows [0, cnt) of the destination must be bit copies of the source rows at idx_gpu."""
     cnt = idx_gpu.size
     sel = torch.from_numpy(idx_gpu.astype(np.int64))
-    assert torch.equal(k_out[:cnt].cpu().view(torch.int16), ref["k"][sel].view(torch.int16))
+    bits = torch.uint8 if ref["k"].dtype == torch.float8_e4m3fn else torch.int16
+    assert torch.equal(k_out[:cnt].cpu().view(bits), ref["k"].view(bits)[sel])
     if v_out is not None:
-        assert torch.equal(v_out[:cnt].cpu().view(torch.int16), ref["v"][sel].view(torch.int16))
+        assert torch.equal(v_out[:cnt].cpu().view(bits), ref["v"].view(bits)[sel])
     if pos_out is not None:
         assert torch.equal(pos_out[:cnt].cpu().long(), ref["pos"][sel])
         assert torch.all(pos_out[1:cnt] > pos_out[:cnt - 1])

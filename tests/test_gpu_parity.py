@@ -976,3 +976,45 @@ def test_fused_selection_of_long_units_equals_the_two_step_path(G, ties):
         assert torch.equal(idx2[0][kept == t].long(), eq[: int((kept == t).sum())])     # the lowest slots of the group
     else:
         check_unit(w, res, oracle_unit(w, 0, 0, 1, sp.budget), 0, 0, 1, sp.budget)
+
+
+def _as_e4m3(w):
+    """The same workload with K and V rounded to e4m3 (k_kind 3)."""
+    return W.Workload(w.spec, w.q_center, w.q_mean_norm, w.k.float().to(torch.float8_e4m3fn), w.v.float().to(torch.float8_e4m3fn),
+                      w.seq_lens, w.cur_pos, w.positions, w.page_table)
+
+
+@pytest.mark.parametrize("shape", ["g4", "g8_paged_in_place", "g16", "g3_half_split", "g1_long"])
+def test_e4m3_keys(shape):
+    """8-bit caches (k_kind 3): raw and final scores, kept slots and the copied 128-byte K and V rows of every unit
+    against the oracle's reading of the same bytes: 16-key tiles with a ragged tail, one, two and four MMA column
+    tiles (G = 1..16), both band layouts, paged keys compacted in place, and a unit long enough for the one-sweep
+    selection."""
+    base = W.SPECS["qwen3_8b_oneshot_32k"]
+    layout, in_place = 0, False
+    if shape == "g4":
+        sp = base.scaled(name="e4_g4", n_layers=2, n_kv_heads=2, n_keys=5003, budget=400)
+    elif shape == "g8_paged_in_place":
+        sp = W.SPECS["qwen3_32b_ragged_paged"].scaled(name="e4_g8", n_layers=2, n_kv_heads=2, n_seqs=3, n_keys=4000,
+                                                      n_keys_min=300, budget=512)
+        in_place = True
+    elif shape == "g16":
+        sp = base.scaled(name="e4_g16", n_layers=1, n_kv_heads=1, group_size=16, n_keys=3000, budget=300)
+    elif shape == "g3_half_split":
+        sp = base.scaled(name="e4_g3", n_layers=1, n_kv_heads=2, group_size=3, n_keys=3333, budget=200)
+        layout = 1
+    else:
+        sp = base.scaled(name="e4_g1", n_layers=1, n_kv_heads=1, group_size=1, n_keys=70001, budget=1000)
+    w = W.make_workload(sp, DEV)
+    if layout == 1:
+        perm = torch.cat([torch.arange(0, 128, 2), torch.arange(1, 128, 2)])
+        w = W.Workload(sp, w.q_center[..., perm].contiguous(), w.q_mean_norm, w.k[..., perm.to(DEV)].contiguous(),
+                       w.v, w.seq_lens, w.cur_pos, None, None)
+    w = _as_e4m3(w)
+    units = _all_units(w)
+    refs = {u: oracle_unit(w, *u, sp.budget, layout=layout) for u in units}      # before any in-place write
+    ctx = make_ctx(w, pair_layout=layout)
+    res = run_compress(w, sp.budget, ctx=ctx, in_place=in_place)
+    assert int(res["status"].item()) == 0
+    for u in units:
+        check_unit(w, res, refs[u], *u, sp.budget)

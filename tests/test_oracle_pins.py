@@ -311,6 +311,40 @@ def test_unit_bf16_chains_the_steps(rng):
     assert np.array_equal(idx, oracle.select(s2, B))
 
 
+def test_e4m3_values_and_the_unit_entry_point(rng):
+    """8-bit keys: the decoder against the format's definition (1.0, the largest finite value 448, the smallest
+    subnormal 2^-9, the smallest normal 2^-6, signs, both zeros, the two not-a-number codes), against torch's own
+    conversion of all 256 codes, and monotone over the positive codes; the whole-unit entry point equals the steps
+    on the decoded values, and equals the bf16 entry point on keys both formats hold exactly."""
+    import torch
+    from paper_2604_04921_b200.workloads import rope_forward, bf16_bits
+    codes = np.arange(256, dtype=np.uint8)
+    val = oracle.e4m3_to_f64(codes)
+    want = {0x38: 1.0, 0x7E: 448.0, 0x01: 2.0 ** -9, 0x08: 2.0 ** -6, 0xB8: -1.0, 0x40: 2.0, 0x3C: 1.5, 0x00: 0.0, 0x07: 7 * 2.0 ** -9}
+    for code, v in want.items():
+        assert val[code] == v, (hex(code), val[code])
+    assert np.signbit(val[0x80]) and val[0x80] == 0.0 and np.isnan(val[0x7F]) and np.isnan(val[0xFF])
+    assert np.all(np.diff(val[:0x7F]) > 0) and np.array_equal(val[0x80:0xFF], -val[:0x7F])
+    lib = torch.from_numpy(codes).view(torch.float8_e4m3fn).double().numpy()
+    assert np.array_equal(np.isnan(val), np.isnan(lib)) and np.array_equal(val[~np.isnan(val)], lib[~np.isnan(lib)])
+    N, G, B = 200, 3, 30
+    g = torch.Generator().manual_seed(3)
+    k = torch.randn(N, D, generator=g, dtype=torch.float64) * 0.5 + torch.randn(D, generator=g, dtype=torch.float64)
+    pos = torch.arange(N)
+    k8 = rope_forward(k, pos, THETA).float().to(torch.float8_e4m3fn)
+    bits8 = k8.view(torch.uint8).numpy()
+    c = rng.standard_normal((G, D))
+    n_mean = band_abs(c) + 0.2
+    raw, s, idx = oracle.unit_e4m3(bits8, pos.numpy(), N, c, n_mean, B)
+    kpre = oracle.unrotate(oracle.e4m3_to_f64(bits8), pos.numpy(), THETA)
+    assert np.max(np.abs(kpre - k.numpy())) < 0.3            # e4m3 rounding only (3 mantissa bits)
+    raw2 = oracle.score_raw(kpre, pos.numpy(), N, c, n_mean)
+    assert np.array_equal(raw, raw2)
+    assert np.array_equal(idx, oracle.select(oracle.normalize(raw2)[1], B))
+    raw_b, s_b, idx_b = oracle.unit_bf16(bf16_bits(k8.to(torch.bfloat16)), pos.numpy(), N, c, n_mean, B)   # exact widening
+    assert np.array_equal(raw, raw_b) and np.array_equal(s, s_b) and np.array_equal(idx, idx_b)
+
+
 def test_calibration_statistics_pins(rng):
     """E[q_f], E|q_f| and R_f against closed forms and an independent computation."""
     T = 360
