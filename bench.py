@@ -136,11 +136,12 @@ class ClockSampler:
             self.proc.kill()
 
 
-def algorithmic_bytes(seq_lens, units_per_seq, budget):
-    """256 N (stream K) + 1036 min(B, N) (re-read kept K, read kept V, write both, idx + positions)."""
+def algorithmic_bytes(seq_lens, units_per_seq, budget, row_bytes=256):
+    """256 N (stream K) + 1036 min(B, N) (re-read kept K, read kept V, write both, idx + positions); rows of
+    row_bytes bytes in general: row_bytes N + (4 row_bytes + 12) min(B, N)."""
     tot = 0
     for n in seq_lens:
-        tot += units_per_seq * (256 * n + 1036 * min(budget, n))
+        tot += units_per_seq * (row_bytes * n + (4 * row_bytes + 12) * min(budget, n))
     return tot
 
 
@@ -285,12 +286,17 @@ def run_calibration(args):
 class Round:
     """One workload resident on the device with everything a timed tri_compress step needs."""
 
-    def __init__(self, spec, L, dev, pre_rope=False):
+    def __init__(self, spec, L, dev, pre_rope=False, e4m3=False):
         import torch
         from paper_2604_04921_b200 import binding as tb
         from paper_2604_04921_b200 import workloads as W
         self.spec, self.L, self.dev = spec, L, dev
         self.w = w = W.make_workload(spec, dev, layer0=0, n_layers=L)
+        self.row_bytes = 256
+        if e4m3:
+            # the same rows rounded to e4m3 (k_kind 3): 128-byte K and V rows
+            w.k, w.v = w.k.float().to(torch.float8_e4m3fn), w.v.float().to(torch.float8_e4m3fn)
+            self.row_bytes = 128
         S, H, G, B = spec.n_seqs, spec.n_kv_heads, spec.group_size, spec.budget
         self.ctx = tb.TriContext(L, H, G, w.q_center, w.q_mean_norm, rope_theta=spec.theta)
         # pre_rope: the same bf16 rows read as pre-RoPE vectors (k_kind 2): the kernels' work does not depend on the values
@@ -302,7 +308,7 @@ class Round:
             self.dst = tb.CacheView(w.k, w.v, page_table=w.page_table, n_max=self.n_max, pre_rope=pre_rope)
             self.k2 = self.v2 = self.p2 = None
         else:
-            self.k2 = torch.empty(L, S, H, B, 128, dtype=torch.bfloat16, device=dev)
+            self.k2 = torch.empty(L, S, H, B, 128, dtype=w.k.dtype, device=dev)
             self.v2 = torch.empty_like(self.k2)
             self.p2 = torch.empty(L, S, H, B, dtype=torch.int32, device=dev)
             self.dst = tb.CacheView(self.k2, self.v2, positions=self.p2, pre_rope=pre_rope)
@@ -310,7 +316,7 @@ class Round:
         self.kept_cnt = torch.zeros(self.U, dtype=torch.int32, device=dev)
         self.lens = w.seq_lens.tolist()
         self.keys_per_step = sum(self.lens) * L * H
-        self.abytes = algorithmic_bytes(self.lens, L * H, B)
+        self.abytes = algorithmic_bytes(self.lens, L * H, B, self.row_bytes)
         self.launches_per_step = self.ctx.compress_launches(self.src, S, self.dst)
         # An in-place round changes its own input (the kept rows move to the front of each sequence's pages), and
         # a second round on that state would find nearly every kept row already in place.  So for the paged
@@ -374,7 +380,7 @@ class Round:
 
     def hbm(self, ms_step, peak):
         gbs = self.abytes / (ms_step * 1e-3) / 1e9
-        return {"algorithmic_bytes_per_step": self.abytes, "kv_bytes": (self.w.k.numel() + self.w.v.numel()) * 2,
+        return {"algorithmic_bytes_per_step": self.abytes, "kv_bytes": (self.w.k.numel() + self.w.v.numel()) * self.w.k.element_size(),
                 "achieved_gbs": gbs, "frac_of_measured_copy_peak": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS}
 
     def close(self):
@@ -392,6 +398,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="time the headline workload only")
+    ap.add_argument("--e4m3", action="store_true", help="the workload's K and V rounded to e4m3 (k_kind 3: 128-byte rows, f16 tensor-core scoring)")
     ap.add_argument("--pre-rope", action="store_true", help="treat the bf16 keys as pre-RoPE vectors (k_kind 2: fp32 scoring with phasor tables)")
     ap.add_argument("--calibration", action="store_true", help="time the calibration-statistics pass instead of the round")
     ap.add_argument("--tokens", type=int, default=0, help="--calibration: tokens per pass (default 262,144)")
@@ -402,7 +409,7 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
     from paper_2604_04921_b200 import workloads as W
-    others = args.workload is None and args.layers == 0 and not args.no_others and not args.pre_rope
+    others = args.workload is None and args.layers == 0 and not args.no_others and not args.pre_rope and not args.e4m3
     spec = W.SPECS[args.workload or DEFAULT_WORKLOAD]
     if args.impl == "reference":
         run_reference(args, spec)
@@ -446,7 +453,7 @@ def main():
         return n, ms, (sampler.summary(first) if rank == 0 else None)
 
     L = args.layers if args.layers > 0 else spec.n_layers
-    rd = Round(spec, L, dev, pre_rope=args.pre_rope)
+    rd = Round(spec, L, dev, pre_rope=args.pre_rope, e4m3=args.e4m3)
     rd.warm(args.warmup)
     barrier()
     sustained = None
@@ -462,20 +469,23 @@ def main():
                      "hbm": rd.hbm(ms, peak), "clocks": ck}
 
     per = rd.kernel_ms(min(args.steps, 50))
-    score_bytes = 256 * rd.keys_per_step
+    score_bytes = rd.row_bytes * rd.keys_per_step
     score_gbs = score_bytes / (per["score"] * 1e-3) / 1e9
     cfg = workload_config(spec, L, world)
     if args.pre_rope:
         cfg["keys"] = "bf16 pre-RoPE (k_kind 2)"
+    if args.e4m3:
+        cfg["keys"] = "e4m3 post-RoPE keys and e4m3 values (k_kind 3), 128-byte rows"
+        cfg["storage_dtype"] = "e4m3"
     line = {
         "metric": METRIC, "value": whole_job_value(world, rd.keys_per_step, ms_step), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16" if args.e4m3 else "bf16", "data": "synthetic",
         "config": cfg,
         "keys_per_step": rd.keys_per_step,
         "hbm": rd.hbm(ms_step, peak),
-        "roofline": {"kernel": "k_score_bf16_pre" if args.pre_rope else ("k_score_umma" if spec.group_size > 4 else "k_score_tma"), "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(rd.keys_per_step) if (spec.group_size <= 4 and not args.pre_rope) else None, "peak_source": peak_src,
+        "roofline": {"kernel": "k_score_tma<e4m3>" if args.e4m3 else "k_score_bf16_pre" if args.pre_rope else ("k_score_umma" if spec.group_size > 4 else "k_score_tma"), "bound": "hbm", "achieved": score_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": score_gbs / peak, "traffic": score_traffic_per_launch(rd.keys_per_step) if (spec.group_size <= 4 and not args.pre_rope and not args.e4m3) else None, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": score_bytes, "ms_per_launch": per["score"],
                      "note": "per step; a pipelined round issues the scoring as several launches over unit ranges, "
                              "their bytes and durations are summed"},
@@ -488,7 +498,7 @@ def main():
 
     # ---- end to end through tri_compress_host: pinned host buffers, copies inside the timed region ----
     w, S, B, U = rd.w, spec.n_seqs, spec.budget, rd.U
-    if not args.no_e2e and not w.paged:
+    if not args.no_e2e and not w.paged and not args.e4m3:
         e2e_steps = max(2, min(args.steps, 3 if rd.keys_per_step > 2e7 else 5))
         hk = torch.empty(w.k.shape, dtype=w.k.dtype, pin_memory=True).copy_(w.k)
         hv = torch.empty(w.v.shape, dtype=w.v.dtype, pin_memory=True).copy_(w.v)

@@ -605,7 +605,7 @@ bool aliases(const tri_cache_view *a, const tri_cache_view *b)
 // Whether the round compacts bf16 K + V in place: then the gather is two launches (tiled prefix, parallel pass).
 bool two_pass_compaction(const tri_cache_view *src, const tri_cache_view *dst)
 {
-    return aliases(src, dst) && (src->k_kind == 0 || src->k_kind == 2) && src->v && dst->v;
+    return aliases(src, dst) && src->k_kind != 1 && src->v && dst->v;
 }
 
 tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kept_idx, const int32_t *kept_cnt,
@@ -629,13 +629,20 @@ tri_status run_compact(tri_ctx *c, const tri_cache_view *src, const int32_t *kep
         // in place: the prefix whose sources lie inside the destination range goes tile by tile in one block
         // per unit; everything behind it is a hazard-free gather
         if (rows16) {
-            k_compact_inplace_rows<<<U, kInplaceThreads, 0, st>>>(p);
+            k_compact_inplace_rows<2><<<U, kInplaceThreads, 0, st>>>(p);
             k_gather_rows<true><<<grid, kGatherThreads, 0, st>>>(p);
+        } else if (src->k_kind == 3 && p.v_vec != 0) {
+            dim3 grid8(U, (budget + 2 * kFastRowsPerBlock - 1) / (2 * kFastRowsPerBlock));
+            k_compact_inplace_rows<1><<<U, kInplaceThreads, 0, st>>>(p);
+            k_gather_rows<true, 1><<<grid8, kGatherThreads, 0, st>>>(p);
         } else {
             k_compact_inplace_any<<<U, kInplaceThreads, 0, st>>>(p);
         }
     } else if (rows16) {
         k_gather_rows<false><<<grid, kGatherThreads, 0, st>>>(p);
+    } else if (src->k_kind == 3 && p.v_vec != 0) {
+        dim3 grid8(U, (budget + 2 * kFastRowsPerBlock - 1) / (2 * kFastRowsPerBlock));      // 128-byte rows: two slots per warp step
+        k_gather_rows<false, 1><<<grid8, kGatherThreads, 0, st>>>(p);
     } else {
         dim3 grid_any(U, (budget + kGatherRowsPerBlock - 1) / kGatherRowsPerBlock);
         k_gather_any<<<grid_any, kGatherThreads, 0, st>>>(p);

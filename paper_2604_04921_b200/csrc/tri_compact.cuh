@@ -66,32 +66,38 @@ constexpr int kFastIters = 2;
 constexpr int kFastRowsPerBlock = kGatherWarps * kFastRows * kFastIters;
 constexpr int kInplaceRows = 128;       // rows per tile of the in-place schedule
 
-template <bool AFTER_PREFIX>
+// ESZ = bytes per element: 2 = bf16 rows as described; 1 = e4m3 rows of 128 bytes, 8 lanes per row, so a half-warp
+// carries the K and V row of one slot and a warp two slots at a time (16 rows in flight per warp).
+template <bool AFTER_PREFIX, int ESZ = 2>
 __global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const CompactParams p)
 {
+    constexpr int kPieces = 8 * ESZ;                 // 16-byte pieces per row
+    constexpr int kSlots = 16 / kPieces;             // slots a warp moves per step: 1 or 2
+    constexpr int kGroup = kFastRows * kSlots;       // rows in flight per warp
     const int u = p.u0 + blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
     if (!AFTER_PREFIX && blockIdx.y == 0 && threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0)
         p.new_seq_lens[s] = cnt;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int jw = blockIdx.y * kFastRowsPerBlock + warp * (kFastRows * kFastIters);
+    const int jw = blockIdx.y * (kFastRowsPerBlock * kSlots) + warp * (kGroup * kFastIters);
     if (jw >= cnt) return;
     const int32_t *idx = p.kept_idx + (int64_t)u * p.budget;
-    const bool is_v = lane >= 16;
-    const char *sb = (is_v ? p.src.v : p.src.k) + (lane & 15) * 16;
-    char *db = (is_v ? p.dst.v : p.dst.k) + (lane & 15) * 16;
+    const bool is_v = (lane / kPieces) & 1;
+    const int sub = lane / (2 * kPieces);            // which of the step's slots this lane works on
+    const char *sb = (is_v ? p.src.v : p.src.k) + (lane % kPieces) * 16;
+    char *db = (is_v ? p.dst.v : p.dst.k) + (lane % kPieces) * 16;
     const int n_src = p.src.n_max;
 
 #pragma unroll 1
     for (int it = 0; it < kFastIters; ++it) {
-        const int j0 = jw + it * kFastRows;
+        const int j0 = jw + it * kGroup;
         if (j0 >= cnt) break;
-        if (AFTER_PREFIX && __ldg(idx + (j0 & ~(kInplaceRows - 1))) < cnt) continue;   // the first phase moved this tile
+        if (AFTER_PREFIX && __ldg(idx + (j0 & ~(kInplaceRows * kSlots - 1))) < cnt) continue;   // the first phase moved this tile
         // lane r resolves row j0 + r; rows past the count, indices outside the unit and bad page ids are skipped
         int mine = -1;
         int64_t so = -1, dof = -1;
-        if (lane < kFastRows && j0 + lane < cnt) {
+        if (lane < kGroup && j0 + lane < cnt) {
             mine = __ldg(idx + j0 + lane);
             if (mine >= 0 && mine < n_src) {
                 so = row_offset(p.src, l, s, h, mine);
@@ -105,13 +111,13 @@ __global__ void __launch_bounds__(kGatherThreads, 4) k_gather_rows(const Compact
         uint4 val[kFastRows];
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
-            const int64_t o = __shfl_sync(0xffffffffu, so, r);
-            if (o >= 0) val[r] = AFTER_PREFIX ? ld_stream(sb + o * 2) : ld_once(sb + o * 2);   // in place: no read-only path
+            const int64_t o = __shfl_sync(0xffffffffu, so, r * kSlots + sub);
+            if (o >= 0) val[r] = AFTER_PREFIX ? ld_stream(sb + o * ESZ) : ld_once(sb + o * ESZ);   // in place: no read-only path
         }
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
-            const int64_t o = __shfl_sync(0xffffffffu, dof, r);
-            if (o >= 0) st_once(db + o * 2, val[r]);
+            const int64_t o = __shfl_sync(0xffffffffu, dof, r * kSlots + sub);
+            if (o >= 0) st_once(db + o * ESZ, val[r]);
         }
         if (p.dst.positions && mine >= 0)
             p.dst.positions[(int64_t)u * p.dst.n_max + j0 + lane] =
@@ -194,25 +200,29 @@ __global__ void __launch_bounds__(kGatherThreads) k_gather_any(const CompactPara
 constexpr int kInplaceThreads = 512;
 static_assert(kInplaceRows == (kInplaceThreads / 32) * kFastRows, "a tile is 8 rows per warp");
 
+// ESZ as in k_gather_rows: with 128-byte rows a warp holds 16 rows and a tile is 256 rows.
+template <int ESZ = 2>
 __global__ void __launch_bounds__(kInplaceThreads, 2) k_compact_inplace_rows(const CompactParams p)
 {
+    constexpr int kPieces = 8 * ESZ, kSlots = 16 / kPieces, kGroup = kFastRows * kSlots;
     const int u = p.u0 + blockIdx.x;
     const int h = u % p.H, s = (u / p.H) % p.S, l = u / (p.H * p.S);
     const int cnt = min(__ldg(p.kept_cnt + u), p.budget);
     if (threadIdx.x == 0 && p.new_seq_lens && h == 0 && l == 0) p.new_seq_lens[s] = cnt;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int32_t *idx = p.kept_idx + (int64_t)u * p.budget;
-    const bool is_v = lane >= 16;
-    const char *sb = (is_v ? p.src.v : p.src.k) + (lane & 15) * 16;
-    char *db = (is_v ? p.dst.v : p.dst.k) + (lane & 15) * 16;
+    const bool is_v = (lane / kPieces) & 1;
+    const int sub = lane / (2 * kPieces);
+    const char *sb = (is_v ? p.src.v : p.src.k) + (lane % kPieces) * 16;
+    char *db = (is_v ? p.dst.v : p.dst.k) + (lane % kPieces) * 16;
     const int n_src = p.src.n_max;
 
-    for (int t0 = 0; t0 < cnt; t0 += kInplaceRows) {
+    for (int t0 = 0; t0 < cnt; t0 += kInplaceRows * kSlots) {
         if (__ldg(idx + t0) >= cnt) break;                   // the parallel pass takes over from here
-        const int j0 = t0 + warp * kFastRows;
+        const int j0 = t0 + warp * kGroup;
         int mine = -1, pos = 0;
         int64_t so = -1, dof = -1;
-        if (lane < kFastRows && j0 + lane < cnt) {
+        if (lane < kGroup && j0 + lane < cnt) {
             mine = __ldg(idx + j0 + lane);
             if (mine == j0 + lane) {
                 mine = -1;                                   // already in its slot
@@ -232,14 +242,14 @@ __global__ void __launch_bounds__(kInplaceThreads, 2) k_compact_inplace_rows(con
         uint4 val[kFastRows];
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
-            const int64_t o = __shfl_sync(0xffffffffu, so, r);
-            if (o >= 0) val[r] = ld_stream(sb + o * 2);
+            const int64_t o = __shfl_sync(0xffffffffu, so, r * kSlots + sub);
+            if (o >= 0) val[r] = ld_stream(sb + o * ESZ);
         }
         __syncthreads();                                     // every source of the tile has been read
 #pragma unroll
         for (int r = 0; r < kFastRows; ++r) {
-            const int64_t o = __shfl_sync(0xffffffffu, dof, r);
-            if (o >= 0) *reinterpret_cast<uint4 *>(db + o * 2) = val[r];
+            const int64_t o = __shfl_sync(0xffffffffu, dof, r * kSlots + sub);
+            if (o >= 0) *reinterpret_cast<uint4 *>(db + o * ESZ) = val[r];
         }
         if (p.dst.positions && mine >= 0) p.dst.positions[(int64_t)u * p.dst.n_max + j0 + lane] = pos;
     }
