@@ -96,3 +96,21 @@ def test_calibration_rejects_bad_arguments():
     assert L.tri_calib_reset(None, 4, None) == 1
     assert L.tri_calib_finalize(st.data_ptr(), 4, 2, q.data_ptr(), q.data_ptr(), None, None) == 1
     torch.cuda.synchronize()
+
+
+def test_calibration_at_rotary_width_64():
+    """Heads with a 64-wide rotary part (the MLA-style models of the paper's cross-architecture appendix): with
+    interleaved pairs two adjacent heads of 64 components are one row of 128 whose 64 bands are the two heads' 32 + 32,
+    so the statistics of `n_heads` narrow heads come out of a pass over `n_heads / 2` wide ones, read as [n_heads][64]
+    centres and [n_heads][32] norms and mean resultant lengths.  Against the oracle run on every narrow head alone."""
+    T, H = 9001, 6
+    g = torch.Generator().manual_seed(64)
+    q = (torch.randn(H, 64, generator=g)[None] + 0.5 * torch.randn(T, H, 64, generator=g)).to(torch.bfloat16).to(DEV)
+    cal = tb.Calibrator(H // 2)
+    cal.add(q.view(T, H // 2, 128))
+    qc, qn, r = cal.result()
+    torch.cuda.synchronize()
+    res = [oracle.calibrate(q[:, h].double().cpu().numpy()) for h in range(H)]
+    _check(qc.view(H, 64), np.stack([x[0] for x in res]))
+    _check(qn.view(H, 32), np.stack([x[1] for x in res]))
+    _check(r.view(H, 32), np.stack([x[2] for x in res]))
