@@ -243,6 +243,25 @@ k_score_umma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
 
     if (warp == kUComputeWarps) {
         // ---------------- producer ----------------
+        // lane (2 sub + half) copies one 16-row box of a tile.  Where its box of tile t lies (for paged keys a page-table
+        // entry) is looked up one tile ahead, so that the lookup's latency is spent under the wait for the stage, not after it
+        const int sub = lane >> 1, half = lane & 1;
+        auto locate = [&](int t, int &c1, int &c3) {
+            const int row = key_begin + t * kUTile + sub * kTileKeys;
+            c1 = row; c3 = s;
+            if (p.src.paged && t < ntiles && row < key_end) {
+                const int pg = p.src.page_shift >= 0 ? row >> p.src.page_shift : row / p.src.page_size;
+                int page = __ldg(p.src.page_table + (int64_t)s * p.src.max_pages_per_seq + pg);
+                if (p.src.n_pages > 0 && (page < 0 || page >= p.src.n_pages)) {
+                    if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
+                    page = 0;                      // stay inside the pool; the unit's output is unspecified
+                }
+                c1 = row - pg * p.src.page_size;
+                c3 = page;
+            }
+        };
+        int c1, c3;
+        locate(0, c1, c3);
         for (int t = 0; t < ntiles; ++t) {
             const int st = t % kUStages;
             bool ok = t < kUStages || mbar_wait_parked(b_kempty + 8 * st, ((t / kUStages) - 1) & 1);
@@ -252,23 +271,10 @@ k_score_umma(const __grid_constant__ CUtensorMap tmap, const ScoreParams p)
             const int nsub = min(kUTile / kTileKeys, (key_end - row0 + kTileKeys - 1) / kTileKeys);
             if (lane == 0) mbar_expect_tx(b_kfull + 8 * st, (uint32_t)nsub * kTileBytes);
             __syncwarp();
-            if (lane < 2 * nsub) {
-                const int sub = lane >> 1, half = lane & 1;
-                const int row = row0 + sub * kTileKeys;
-                int c1 = row, c3 = s;
-                if (p.src.paged) {
-                    const int pg = p.src.page_shift >= 0 ? row >> p.src.page_shift : row / p.src.page_size;
-                    int page = __ldg(p.src.page_table + (int64_t)s * p.src.max_pages_per_seq + pg);
-                    if (p.src.n_pages > 0 && (page < 0 || page >= p.src.n_pages)) {
-                        if (p.device_status) atomicExch(p.device_status, (int)TRI_ERR_DEVICE_CHECK);
-                        page = 0;                      // stay inside the pool; the unit's output is unspecified
-                    }
-                    c1 = row - pg * p.src.page_size;
-                    c3 = page;
-                }
+            if (lane < 2 * nsub)
                 tma_load_5d(sm_k + st * kUTileBytes + half * kUBlockBytes + sub * (kTileKeys * 128), &tmap, b_kfull + 8 * st,
                             half * (kHeadDim / 2), c1, h, c3, l);
-            }
+            locate(t + 1, c1, c3);
         }
     } else if (warp == kUComputeWarps + 1) {
         // ---------------- MMA issue ----------------
